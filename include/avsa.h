@@ -1,0 +1,140 @@
+/*
+ * avsa -- protected sparse video attention for joint audio-video diffusion transformers, sm_100a.
+ *
+ * C ABI of libavsa.so.  Three calls make one layer-step of the path:
+ *
+ *   avsa_cross_attn_scores   audio->video cross-attention (Eq. 1) that also emits the per-video-token
+ *                            cross-modal response scores (Eq. 2, with the blend of Eq. 4 folded in)
+ *   avsa_build_block_mask    protected token set (Eq. 3 / Eq. 8), block-importance top-k, and the
+ *                            protected block mask (Eq. 9) as ascending per-row column lists
+ *   avsa_sparse_self_attn    video self-attention under that mask (Eq. 10 / Eq. 11)
+ *
+ * Conventions for every call
+ *   - All data pointers are DEVICE pointers unless a parameter says "host".  The caller owns every
+ *     buffer.  The library allocates no device memory, never synchronises the stream (except
+ *     avsa_read_status) and enqueues work on the given stream only.
+ *   - Tensors are bf16 with the head dimension contiguous, described by element strides (avsa_bf16_4d),
+ *     so both [B,H,N,d] and [B,N,H,d] storage work.  Base pointers must be 16-byte aligned and strides
+ *     multiples of 8 elements.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *   - `ws` is scratch of at least the matching *_workspace_bytes(); its first 16 bytes are a status
+ *     record the kernels fill when a device-side check fails (a wait that ran out of time, or a
+ *     malformed column list).  Calls on the same workspace must not overlap on the GPU.
+ *   - Errors detectable on the host return at once with nothing enqueued.  Return values are
+ *     avsa_status codes.
+ *   - Supported shapes: (blk, d) in {(128,128), (64,64)}; any N >= 1 (the last block may be partial:
+ *     pooled means divide by the valid count, invalid keys are masked, rows >= N are not written).
+ */
+#ifndef AVSA_H_
+#define AVSA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define AVSA_API __attribute__((visibility("default")))
+#else
+#define AVSA_API
+#endif
+
+typedef enum {
+  AVSA_OK = 0,
+  AVSA_ERR_INVALID_ARG = 1,  /* null pointer, bad size, bad alignment or stride */
+  AVSA_ERR_UNSUPPORTED = 2,  /* (blk, d) combination or device not supported */
+  AVSA_ERR_WORKSPACE = 3,    /* ws is NULL or smaller than *_workspace_bytes() */
+  AVSA_ERR_CUDA = 4,         /* a CUDA runtime / driver call failed */
+  AVSA_ERR_TIMEOUT = 5,      /* device: a bounded wait expired (read with avsa_read_status) */
+  AVSA_ERR_BAD_MASK = 6      /* device: a column list entry was out of range or not ascending */
+} avsa_status;
+
+/* bf16 tensor [B,H,N,d], d contiguous; strides in elements. */
+typedef struct {
+  const void* ptr;
+  int64_t stride_b, stride_h, stride_n;
+} avsa_bf16_4d;
+
+/* flags of avsa_build_block_mask */
+#define AVSA_PROTECT_ROWS 1u            /* Eq. 9: a protected query block keeps every key block */
+#define AVSA_PROTECT_COLS 2u            /* opt-in superset: protected key blocks visible to all rows */
+#define AVSA_USE_GIVEN_BLOCK_SCORES 4u  /* block_scores is an input; q and k are not read */
+
+/*
+ * (1) Cross-attention with response scores -- Eq. 1, Eq. 2 (and the running blend of Eq. 4).
+ *
+ *   A[b,h,j,i] = softmax_i(q[b,h,j,:] . k[b,h,i,:] * softmax_scale)            (queries j, keys i)
+ *   o[b,h,j,:] = sum_i A[b,h,j,i] v[b,h,i,:]                  -> o   bf16, same strides as q's tensor
+ *   lse[b,h,j] = natural-log log-sum-exp of row j              -> lse fp32 [B,H,Nq]
+ *   scores[b,i] = score_beta * scores[b,i] + score_gamma * sum_h sum_j A[b,h,j,i]   fp32 [B,Nk]
+ *
+ * For the audio->video direction q holds the audio queries and k, v the video keys/values.  The
+ * paper's Norm is any scalar: score_gamma = 1/(H*Nq*layers) makes the scores sum to 1; score_beta = 1
+ * accumulates layers; score_beta = alpha with score_gamma = (1-alpha)/(H*Nq) is Eq. 4.
+ * With score_beta == 0 the previous contents of scores are ignored (may be uninitialised).
+ * o, lse and scores may each be NULL to skip that output (scores == NULL skips the second pass).
+ * softmax_scale == 0 means 1/sqrt(d).  Nq <= 512.  The head sum is taken in a fixed order, so
+ * results reproduce bit for bit.  `o` has strides (o_stride_b, o_stride_h, o_stride_n) = q's.
+ */
+AVSA_API int avsa_cross_attn_scores(int B, int H, int Nq, int Nk, int d, avsa_bf16_4d q, avsa_bf16_4d k, avsa_bf16_4d v,
+                           void* o_bf16, float* lse, float* scores, float score_beta, float score_gamma,
+                           float softmax_scale, void* ws, size_t ws_bytes, void* stream);
+AVSA_API size_t avsa_cross_attn_scores_workspace_bytes(int B, int H, int Nq, int Nk, int d);
+
+/*
+ * (2) Mask construction -- Eq. 3 / Eq. 8 (protected set), Eq. 9 (protected mask), and the base
+ * sparse pattern the paper leaves open, here: block mean-pooling of q and k, block scores
+ * Bs[b,h,qb,kb] = mean(q block qb) . mean(k block kb) * softmax_scale, per (head, query block)
+ * top-k_keep over kb.
+ *
+ *   scores       fp32 [B,N] token saliency; may be NULL iff n_protect == 0
+ *   n_protect    size of the protected token set, 0 <= n_protect <= N (= ceil(rho N), host integer)
+ *   k_keep       kept key blocks per unprotected row, 1 <= k_keep <= NB, NB = ceil(N / blk)
+ *   block_scores fp32 [B,H,NB,NB]: output, or input with AVSA_USE_GIVEN_BLOCK_SCORES (never NULL)
+ *   col_idx      int32 [B,H,NB,NB]: kept key blocks of each row, ascending, unused slots = -1
+ *   col_cnt      int32 [B,H,NB]
+ *   prot_tok     uint8 [B,N]  1 = token in the protected set (optional, may be NULL)
+ *   prot_blk     uint8 [B,NB] 1 = block holds a protected token (optional, may be NULL)
+ *
+ * Every top-k orders by (value larger, then index smaller); NaN ranks as -inf; -0 equals +0.
+ * Given the same fp32 scores / block_scores the outputs are exactly determined (integer results).
+ * flags == 0 is treated as AVSA_PROTECT_ROWS.  NB <= 2048.
+ */
+AVSA_API int avsa_build_block_mask(int B, int H, int N, int d, int blk, avsa_bf16_4d q, avsa_bf16_4d k, const float* scores,
+                          int n_protect, int k_keep, unsigned flags, float softmax_scale, float* block_scores,
+                          int32_t* col_idx, int32_t* col_cnt, uint8_t* prot_tok, uint8_t* prot_blk, void* ws,
+                          size_t ws_bytes, void* stream);
+AVSA_API size_t avsa_build_block_mask_workspace_bytes(int B, int H, int N, int d, int blk);
+
+/*
+ * (3) Block-sparse self-attention -- Eq. 10 (Eq. 5 when every list is full).
+ *
+ *   o[b,h,i,:] = softmax_j(q_i . k_j * softmax_scale  restricted to keys j of the listed blocks) v
+ *
+ * For query block qb of head h the kept key blocks are col_idx[b,h,qb,0 .. col_cnt[b,h,qb]-1]
+ * (row stride NB, ascending, each in [0,NB)).  Every list needs at least one entry; a malformed
+ * entry sets AVSA_ERR_BAD_MASK in the status record and that block is skipped without any
+ * out-of-range access.  o is bf16 with the strides of q; lse (optional) is fp32 [B,H,N] natural log.
+ */
+AVSA_API int avsa_sparse_self_attn(int B, int H, int N, int d, int blk, avsa_bf16_4d q, avsa_bf16_4d k, avsa_bf16_4d v,
+                          const int32_t* col_idx, const int32_t* col_cnt, void* o_bf16, float* lse,
+                          float softmax_scale, void* ws, size_t ws_bytes, void* stream);
+AVSA_API size_t avsa_sparse_self_attn_workspace_bytes(int B, int H, int N, int d, int blk);
+
+/* Host integer ceil(pct/100 * n): the count forms of rho and kappa (Eq. 8's ceiling). */
+AVSA_API int avsa_count_from_percent(int pct, int n);
+
+/* Synchronises `stream`, copies the status record of `ws` to the host and returns its code
+ * (AVSA_OK, AVSA_ERR_TIMEOUT or AVSA_ERR_BAD_MASK).  detail (host, optional) receives 3 ints that
+ * say where the check failed.  For tests and debugging; the hot path never calls it. */
+AVSA_API int avsa_read_status(const void* ws, void* stream, int* detail);
+
+AVSA_API const char* avsa_status_string(int status);
+AVSA_API int avsa_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* AVSA_H_ */

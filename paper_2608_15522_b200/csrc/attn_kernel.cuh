@@ -1,0 +1,384 @@
+// Flash-attention forward tile kernel for sm_100a, shared by the block-sparse self-attention
+// (Eq. 10) and the first pass of the cross-attention (Eq. 1).
+//
+// One CTA per work item = one query tile and a list of key tiles.  Warp roles:
+//   warp 0      TMA producer: Q tile once, then the listed K and V tiles through two 3-stage rings
+//   warp 1      MMA issuer: S = Q K^T (operands in shared memory) and O += P V (P in tensor memory)
+//   warp 2      tensor-memory allocation
+//   warps 4-7   softmax group 0: even tiles of the list, accumulator O0
+//   warps 8-11  softmax group 1: odd tiles of the list, accumulator O1
+// The two groups keep independent running maxima / sums; the epilogue merges (O0, m0, l0) and
+// (O1, m1, l1) exactly as a two-way split of the key axis.
+// Tensor memory: S0 | S1 | O0 | O1, 128 columns each; P (bf16) overwrites the front of its S buffer.
+//
+// MODE_LIST   key tiles come from an explicit ascending list; the output tile is converted to bf16
+//             and TMA-stored; optional natural-log LSE.
+// MODE_RANGE  key tiles are a contiguous range (one split of the key axis); the output is a partial
+//             result (fp32 rows normalised by their own sum, plus the log2-domain LSE of the split).
+#pragma once
+#include "avsa_common.cuh"
+#include "sm100_ptx.cuh"
+
+namespace avsa {
+
+constexpr int kAttnThreads = 384;
+constexpr int kStages = 3;
+constexpr float kRescaleThreshold = 8.0f;   // log2 units: O is rescaled only when a row max grew by more
+
+enum { MODE_LIST = 0, MODE_RANGE = 1 };
+
+enum AttnWhere {
+  kWhereQFull = 1, kWhereKEmpty, kWhereVEmpty, kWhereKFull, kWhereVFull, kWherePFull, kWhereSFull, kWhereFinal,
+  kWhereSmemAlign, kWhereList
+};
+
+template <int BLK, int D>
+struct AttnSmem {
+  static constexpr int kTileBytes = BLK * D * 2;
+  static constexpr int kQBytes = 128 * D * 2;        // 128 MMA rows; only BLK of them are loaded
+  static constexpr int kQ = 0;
+  static constexpr int kK = kQBytes;
+  static constexpr int kV = kK + kStages * kTileBytes;
+  static constexpr int kBars = kV + kStages * kTileBytes;
+  static constexpr int kNumBars = 1 + 4 * kStages + 2 + 2 + 1;
+  static constexpr int kStats = kBars + kNumBars * 8;          // float [2][2][128]: m, l per group and row
+  static constexpr int kMisc = kStats + 2 * 2 * 128 * 4;       // tmem base, abort flag
+  static constexpr int kTotal = kMisc + 16;
+};
+
+struct AttnParams {
+  // MODE_LIST
+  const int32_t* col_idx;   // [B,H,NB,NB]
+  const int32_t* col_cnt;   // [B,H,NB]
+  float* lse;               // [B,H,Nq] natural log, optional
+  // MODE_RANGE
+  float* part_o;            // [items][BLK][D] fp32
+  float* part_lse2;         // [items][BLK]
+  int n_split, tiles_per_split;
+  // both
+  StatusRecord* status;
+  int H;
+  int Nq, NQT;              // query rows and query tiles
+  int Nk, NKB;              // key rows and key tiles
+  float scale_log2;         // softmax_scale * log2(e)
+};
+
+template <int BLK, int D, int MODE>
+__global__ void __launch_bounds__(kAttnThreads, 1)
+attn_fwd_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUtensorMap tmk,
+                const __grid_constant__ CUtensorMap tmv, const __grid_constant__ CUtensorMap tmo,
+                const AttnParams p) {
+  using L = AttnSmem<BLK, D>;
+  constexpr int NPANEL = D / 64;
+  constexpr int PANEL_BYTES = BLK * 128;        // one 64-channel panel of a K/V tile
+  constexpr int QPANEL_BYTES = 128 * 128;
+  extern __shared__ __align__(1024) uint8_t smem[];
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int h = blockIdx.y, b = blockIdx.z;
+  int qt, split = 0, kb0 = 0, cnt;
+  const int32_t* list = nullptr;
+  if (MODE == MODE_LIST) {
+    qt = blockIdx.x;
+    const int row_id = (b * p.H + h) * p.NQT + qt;
+    list = p.col_idx + static_cast<int64_t>(row_id) * p.NKB;
+    cnt = p.col_cnt[row_id];
+  } else {
+    qt = blockIdx.x / p.n_split;
+    split = blockIdx.x % p.n_split;
+    kb0 = split * p.tiles_per_split;
+    cnt = min(p.NKB, kb0 + p.tiles_per_split) - kb0;
+  }
+  const int item = ((b * p.H + h) * p.NQT + qt) * (MODE == MODE_LIST ? 1 : p.n_split) + split;
+
+  // ---- validation: nothing is loaded through a bad list entry
+  {
+    int bad = (cnt < 1 || cnt > p.NKB) ? 1 : 0;
+    if (MODE == MODE_LIST) {
+      const int n = min(max(cnt, 0), p.NKB);
+      for (int t = tid; t < n; t += kAttnThreads) {
+        const int kb = list[t];
+        const int prev = t > 0 ? list[t - 1] : -1;
+        if (kb < 0 || kb >= p.NKB || kb <= prev) bad = 1;
+      }
+    }
+    const bool misaligned = (smem_u32(smem) & 1023u) != 0u;
+    if (misaligned) bad = 1;
+    const int any_bad = __syncthreads_or(bad);
+    if (any_bad) {
+      if (tid == 0)
+        report_status(p.status, misaligned ? AVSA_ERR_CUDA : AVSA_ERR_BAD_MASK, misaligned ? kWhereSmemAlign : kWhereList,
+                      item, cnt);
+      return;
+    }
+  }
+
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::kBars);
+  const uint32_t bar0 = smem_u32(bars);
+  auto BAR = [&](int i) { return bar0 + static_cast<uint32_t>(i) * 8u; };
+  constexpr int Q_FULL = 0, K_FULL = 1, K_EMPTY = 1 + kStages, V_FULL = 1 + 2 * kStages, V_EMPTY = 1 + 3 * kStages,
+                S_FULL = 1 + 4 * kStages, P_FULL = S_FULL + 2, FINAL = P_FULL + 2;
+  float* stats = reinterpret_cast<float*>(smem + L::kStats);
+  volatile uint32_t* misc = reinterpret_cast<volatile uint32_t*>(smem + L::kMisc);   // [0] tmem base, [1] abort
+
+  if (tid == 0) {
+    mbar_init(BAR(Q_FULL), 1);
+    for (int s = 0; s < kStages; s++) {
+      mbar_init(BAR(K_FULL + s), 1);
+      mbar_init(BAR(K_EMPTY + s), 1);
+      mbar_init(BAR(V_FULL + s), 1);
+      mbar_init(BAR(V_EMPTY + s), 1);
+    }
+    for (int w = 0; w < 2; w++) {
+      mbar_init(BAR(S_FULL + w), 1);
+      mbar_init(BAR(P_FULL + w), 128);
+    }
+    mbar_init(BAR(FINAL), 1);
+    misc[1] = 0u;
+    fence_mbar_init();
+    prefetch_tmap(&tmq);
+    prefetch_tmap(&tmk);
+    prefetch_tmap(&tmv);
+    if (MODE == MODE_LIST) prefetch_tmap(&tmo);
+  }
+  if (warp == 2) {
+    tmem_alloc(smem_u32(smem + L::kMisc), 512);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = misc[0];
+  const uint32_t TM_S[2] = {tmem + 0u, tmem + 128u};
+  const uint32_t TM_O[2] = {tmem + 256u, tmem + 384u};
+
+  // A wait that gives up: records where, raises the CTA-wide abort flag, and lets every role unwind.
+  auto wait_or_abort = [&](int bar, uint32_t parity, int where, int tile) -> bool {
+    if (misc[1] != 0u) return false;
+    if (mbar_wait(BAR(bar), parity)) return true;
+    report_status(p.status, AVSA_ERR_TIMEOUT, where, item, tile);
+    misc[1] = 1u;
+    return false;
+  };
+
+  const int n_tiles[2] = {(cnt + 1) >> 1, cnt >> 1};
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      mbar_expect_tx(BAR(Q_FULL), BLK * D * 2);
+      for (int pn = 0; pn < NPANEL; pn++)
+        tma_load_4d(smem_u32(smem + L::kQ) + pn * QPANEL_BYTES, &tmq, BAR(Q_FULL), pn * 64, qt * BLK, h, b);
+    }
+    for (int t0 = 0; t0 < cnt; t0 += 32) {
+      int mine = kb0 + t0 + lane;
+      if (MODE == MODE_LIST) mine = (t0 + lane < cnt) ? list[t0 + lane] : 0;
+      const int nn = min(32, cnt - t0);
+      for (int j = 0; j < nn; j++) {
+        const int kb = __shfl_sync(0xffffffffu, mine, j);
+        if (lane == 0) {
+          const int t = t0 + j, s = t % kStages, f = t / kStages;
+          bool ok = true;
+          if (f > 0) ok = wait_or_abort(K_EMPTY + s, (f - 1) & 1, kWhereKEmpty, t);
+          if (ok) {
+            mbar_expect_tx(BAR(K_FULL + s), L::kTileBytes);
+            for (int pn = 0; pn < NPANEL; pn++)
+              tma_load_4d(smem_u32(smem + L::kK) + s * L::kTileBytes + pn * PANEL_BYTES, &tmk, BAR(K_FULL + s), pn * 64,
+                          kb * BLK, h, b);
+          }
+          if (ok && f > 0) ok = wait_or_abort(V_EMPTY + s, (f - 1) & 1, kWhereVEmpty, t);
+          if (ok) {
+            mbar_expect_tx(BAR(V_FULL + s), L::kTileBytes);
+            for (int pn = 0; pn < NPANEL; pn++)
+              tma_load_4d(smem_u32(smem + L::kV) + s * L::kTileBytes + pn * PANEL_BYTES, &tmv, BAR(V_FULL + s), pn * 64,
+                          kb * BLK, h, b);
+          }
+        }
+      }
+      if (__any_sync(0xffffffffu, misc[1] != 0u)) break;
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      const uint32_t idesc_qk = make_idesc_bf16(128, BLK, 0, 0);
+      const uint32_t idesc_pv = make_idesc_bf16(128, D, 0, 1);
+      const uint32_t q_addr = smem_u32(smem + L::kQ);
+      bool ok = wait_or_abort(Q_FULL, 0, kWhereQFull, 0);
+      for (int t = 0; t <= cnt && ok; t++) {
+        if (t < cnt) {
+          const int w = t & 1, s = t % kStages, f = t / kStages;
+          ok = wait_or_abort(K_FULL + s, f & 1, kWhereKFull, t);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t k_addr = smem_u32(smem + L::kK) + s * L::kTileBytes;
+#pragma unroll
+          for (int ks = 0; ks < D / 16; ks++) {
+            const uint64_t ad = make_sdesc(q_addr + (ks >> 2) * QPANEL_BYTES + (ks & 3) * 32, 16, 1024);
+            const uint64_t bd = make_sdesc(k_addr + (ks >> 2) * PANEL_BYTES + (ks & 3) * 32, 16, 1024);
+            umma_ss(TM_S[w], ad, bd, idesc_qk, ks > 0 ? 1u : 0u);
+          }
+          umma_commit(BAR(S_FULL + w));
+          umma_commit(BAR(K_EMPTY + s));
+        }
+        if (t >= 1) {
+          const int u = t - 1, w = u & 1, s = u % kStages, f = u / kStages, i = u >> 1;
+          ok = wait_or_abort(P_FULL + w, i & 1, kWherePFull, u);
+          if (!ok) break;
+          ok = wait_or_abort(V_FULL + s, f & 1, kWhereVFull, u);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t v_addr = smem_u32(smem + L::kV) + s * L::kTileBytes;
+#pragma unroll
+          for (int ks = 0; ks < BLK / 16; ks++) {
+            const uint64_t bd = make_sdesc(v_addr + ks * 2048, PANEL_BYTES, 1024);
+            umma_ts(TM_O[w], TM_S[w] + ks * 8, bd, idesc_pv, (i > 0 || ks > 0) ? 1u : 0u);
+          }
+          umma_commit(BAR(V_EMPTY + s));
+        }
+      }
+      if (ok) umma_commit(BAR(FINAL));
+    }
+  } else if (warp >= 4) {
+    // ------------------------------------------------------------------ softmax groups + epilogue
+    const int w = (warp - 4) >> 2;               // group
+    const int row = ((warp & 3) << 5) + lane;    // row of the tile == TMEM lane
+    const uint32_t lane_off = static_cast<uint32_t>((warp & 3) * 32) << 16;
+    const int nw = n_tiles[w];
+    const int last_kb = (MODE == MODE_LIST) ? list[cnt - 1] : kb0 + cnt - 1;
+    const int ragged_valid = (last_kb == p.NKB - 1) ? (p.Nk - last_kb * BLK) : BLK;   // valid keys of the last tile
+    float m_run = -INFINITY, l_run = 0.f;
+    bool ok = true;
+    for (int i = 0; i < nw && ok; i++) {
+      const int t = 2 * i + w;
+      ok = wait_or_abort(S_FULL + w, i & 1, kWhereSFull, t);
+      if (!ok) break;
+      tc_fence_after();
+      uint32_t s[BLK];
+#pragma unroll
+      for (int c = 0; c < BLK / 32; c++)
+        tmem_ld32(TM_S[w] + lane_off + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
+      tmem_wait_ld();
+      if (t == cnt - 1 && ragged_valid < BLK) {
+#pragma unroll
+        for (int j = 0; j < BLK; j++)
+          if (j >= ragged_valid) s[j] = 0xff800000u;
+      }
+      float mx = -INFINITY;
+#pragma unroll
+      for (int j = 0; j < BLK; j++) mx = fmaxf(mx, __uint_as_float(s[j]));
+      const float m_new = fmaxf(m_run, mx * p.scale_log2);
+      const bool need = (m_new - m_run) > kRescaleThreshold;     // true on the first tile (m_run = -inf)
+      float factor = 1.f;
+      if (need) {
+        factor = fast_exp2(m_run - m_new);
+        m_run = m_new;
+      }
+      if (i > 0 && __any_sync(0xffffffffu, need)) {
+        // the previous P V of this group has finished (its completion precedes this S): O is stable
+#pragma unroll
+        for (int c = 0; c < D / 32; c++) {
+          uint32_t o[32];
+          tmem_ld32(TM_O[w] + lane_off + c * 32, o);
+          tmem_wait_ld();
+#pragma unroll
+          for (int j = 0; j < 32; j++) o[j] = __float_as_uint(__uint_as_float(o[j]) * factor);
+          tmem_st32(TM_O[w] + lane_off + c * 32, o);
+        }
+      }
+      l_run *= factor;
+      float sum = 0.f;
+      const float neg_m = -m_run;
+#pragma unroll
+      for (int c = 0; c < BLK / 32; c++) {
+        uint32_t pk[16];
+#pragma unroll
+        for (int j = 0; j < 16; j++) {
+          const float p0 = fast_exp2(fmaf(__uint_as_float(s[c * 32 + 2 * j]), p.scale_log2, neg_m));
+          const float p1 = fast_exp2(fmaf(__uint_as_float(s[c * 32 + 2 * j + 1]), p.scale_log2, neg_m));
+          sum += p0 + p1;
+          pk[j] = pack_bf16x2(p0, p1);
+        }
+        tmem_st16(TM_S[w] + lane_off + c * 16, pk);
+      }
+      l_run += sum;
+      tmem_wait_st();
+      tc_fence_before();
+      mbar_arrive(BAR(P_FULL + w));
+    }
+    // publish this group's statistics, then merge the two halves of the key axis
+    stats[(w * 2 + 0) * 128 + row] = m_run;
+    stats[(w * 2 + 1) * 128 + row] = l_run;
+    asm volatile("bar.sync 1, 256;" ::: "memory");
+    ok = wait_or_abort(FINAL, 0, kWhereFinal, cnt);
+    if (ok) {
+      tc_fence_after();
+      const float m0 = stats[0 * 128 + row], l0 = stats[1 * 128 + row];
+      const bool have1 = n_tiles[1] > 0;
+      const float m1 = have1 ? stats[2 * 128 + row] : -INFINITY;
+      const float l1 = have1 ? stats[3 * 128 + row] : 0.f;
+      const float m = fmaxf(m0, m1);
+      const float a0 = fast_exp2(m0 - m), a1 = have1 ? fast_exp2(m1 - m) : 0.f;
+      const float Lsum = a0 * l0 + a1 * l1;
+      const float f0 = a0 / Lsum, f1 = a1 / Lsum;
+      // group w handles channels [w*D/2, (w+1)*D/2) of every row
+      constexpr int HALF = D / 2;
+      uint8_t* stage = smem + L::kQ;     // the Q tile is dead once every MMA has finished
+#pragma unroll
+      for (int c = 0; c < HALF / 32; c++) {
+        const int col0 = w * HALF + c * 32;
+        uint32_t o0[32], o1[32];
+        tmem_ld32(TM_O[0] + lane_off + col0, o0);
+        if (have1) tmem_ld32(TM_O[1] + lane_off + col0, o1);
+        tmem_wait_ld();
+        float v[32];
+#pragma unroll
+        for (int j = 0; j < 32; j++) {
+          v[j] = __uint_as_float(o0[j]) * f0;
+          if (have1) v[j] = fmaf(__uint_as_float(o1[j]), f1, v[j]);
+        }
+        if (row < BLK) {
+          if (MODE == MODE_LIST) {
+#pragma unroll
+            for (int g = 0; g < 4; g++) {
+              const int col = col0 + g * 8;
+              const int panel = col >> 6, chunk = (col & 63) >> 3;
+              uint4 val;
+              val.x = pack_bf16x2(v[g * 8 + 0], v[g * 8 + 1]);
+              val.y = pack_bf16x2(v[g * 8 + 2], v[g * 8 + 3]);
+              val.z = pack_bf16x2(v[g * 8 + 4], v[g * 8 + 5]);
+              val.w = pack_bf16x2(v[g * 8 + 6], v[g * 8 + 7]);
+              *reinterpret_cast<uint4*>(stage + panel * QPANEL_BYTES + row * 128 + ((chunk ^ (row & 7)) << 4)) = val;
+            }
+          } else {
+            float4* dst = reinterpret_cast<float4*>(p.part_o + (static_cast<int64_t>(item) * BLK + row) * D + col0);
+#pragma unroll
+            for (int g = 0; g < 8; g++) dst[g] = make_float4(v[g * 4], v[g * 4 + 1], v[g * 4 + 2], v[g * 4 + 3]);
+          }
+        }
+      }
+      if (w == 0 && row < BLK) {
+        const float lse2 = m + log2f(Lsum);
+        if (MODE == MODE_LIST) {
+          if (p.lse != nullptr && qt * BLK + row < p.Nq)
+            p.lse[(static_cast<int64_t>(b) * p.H + h) * p.Nq + qt * BLK + row] = lse2 * 0.6931471805599453f;
+        } else {
+          p.part_lse2[static_cast<int64_t>(item) * BLK + row] = lse2;
+        }
+      }
+      if (MODE == MODE_LIST) fence_proxy_async();
+    }
+    tc_fence_before();
+    asm volatile("bar.sync 1, 256;" ::: "memory");
+    if (MODE == MODE_LIST && ok && warp == 4 && lane == 0) {
+      for (int pn = 0; pn < NPANEL; pn++)
+        tma_store_4d(&tmo, smem_u32(smem + L::kQ) + pn * QPANEL_BYTES, pn * 64, qt * BLK, h, b);
+      tma_store_commit();
+      tma_store_wait_read();
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 2) tmem_dealloc(tmem, 512);
+}
+
+}  // namespace avsa

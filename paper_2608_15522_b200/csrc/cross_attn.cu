@@ -1,0 +1,393 @@
+// avsa_cross_attn_scores: audio->video cross-attention (Eq. 1) that also emits the per-video-token
+// response scores (Eq. 2), in two passes over the keys.
+//   pass 1  flash attention, key axis split across CTAs -> partial (O, LSE) -> merge -> O, row LSE
+//   pass 2  for every key tile: S^T = K Q^T on the tensor cores, p = exp2(S^T c - lse_j), summed over
+//           the queries -> per-head column sums -> fixed-order head sum with the beta/gamma blend
+#include "attn_kernel.cuh"
+
+namespace avsa {
+
+// ------------------------------------------------------------------------------------------------
+// pass 1 merge: combine the splits of the key axis of every query row
+// ------------------------------------------------------------------------------------------------
+template <int BLK, int D>
+__global__ void __launch_bounds__(128) merge_splits_kernel(const float* __restrict__ part_o,
+                                                           const float* __restrict__ part_lse2, int n_split, int NQT,
+                                                           int Nq, int H, int total_rows, __nv_bfloat16* __restrict__ o,
+                                                           int64_t o_sb, int64_t o_sh, int64_t o_sn,
+                                                           float* __restrict__ lse) {
+  constexpr int TPR = D / 4;
+  const int rg = blockIdx.x * (128 / TPR) + threadIdx.x / TPR;
+  const int c4 = threadIdx.x % TPR;
+  if (rg >= total_rows) return;
+  const int bh = rg / Nq, qrow = rg % Nq;
+  const int qt = qrow / BLK, r = qrow % BLK;
+  const int64_t item0 = (static_cast<int64_t>(bh) * NQT + qt) * n_split;
+  float M = -INFINITY;
+  for (int s = 0; s < n_split; s++) M = fmaxf(M, part_lse2[(item0 + s) * BLK + r]);
+  float W = 0.f;
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int s = 0; s < n_split; s++) {
+    const float w = exp2f(part_lse2[(item0 + s) * BLK + r] - M);
+    const float4 v = *reinterpret_cast<const float4*>(part_o + ((item0 + s) * BLK + r) * D + c4 * 4);
+    W += w;
+    acc.x = fmaf(w, v.x, acc.x);
+    acc.y = fmaf(w, v.y, acc.y);
+    acc.z = fmaf(w, v.z, acc.z);
+    acc.w = fmaf(w, v.w, acc.w);
+  }
+  const float inv = 1.0f / W;
+  if (o != nullptr) {
+    const int b = bh / H, h = bh % H;
+    uint2 pk;
+    pk.x = pack_bf16x2(acc.x * inv, acc.y * inv);
+    pk.y = pack_bf16x2(acc.z * inv, acc.w * inv);
+    *reinterpret_cast<uint2*>(o + b * o_sb + h * o_sh + qrow * o_sn + c4 * 4) = pk;
+  }
+  if (c4 == 0) lse[rg] = (M + log2f(W)) * 0.6931471805599453f;
+}
+
+// ------------------------------------------------------------------------------------------------
+// pass 2: column sums of the attention map.  One CTA keeps the queries of one (batch, head) in
+// shared memory and walks a range of 128-key tiles.  S^T[key, query] accumulates in tensor memory
+// (two buffers of up to 256 columns); two groups of 128 threads (one thread per key row) turn
+// alternate buffers into row sums of exp2(S^T c - lse2[query]).
+//   warp 0 TMA producer, warp 1 MMA issuer, warp 2 tensor-memory allocation,
+//   warps 4-7 / 8-11 the two reduction groups.
+// ------------------------------------------------------------------------------------------------
+constexpr int kColThreads = 384;
+constexpr int kColStages = 3;
+
+struct ColsumParams {
+  const float* lse;        // [B,H,Nq] natural log
+  float* partial;          // [NCH][B,H,Nk]
+  StatusRecord* status;
+  int H, Nq, Nk, NKT;      // NKT = key tiles of 128
+  int NCH, W;              // query chunks and their width (multiple of 16, <= 256)
+  int n_range, tiles_per_range;
+  float scale_log2;
+};
+
+template <int D>
+struct ColsumSmem {
+  static constexpr int kKTile = 128 * D * 2;
+  static constexpr int kK = 0;
+  static constexpr int kQ = kColStages * kKTile;      // NCH * W * D * 2 bytes follow
+  static int bars_offset(int NCH, int W) { return kQ + NCH * W * D * 2; }
+  static constexpr int kNumBars = 1 + 2 * kColStages + 4;
+  static constexpr int kBarBytes = 128;               // keeps the lse table behind it 16-byte aligned
+  static_assert(kNumBars * 8 <= kBarBytes, "barrier area too small");
+  static int total(int NCH, int W) { return bars_offset(NCH, W) + kBarBytes + 512 * 4 + 16; }
+};
+
+enum ColWhere { kColQFull = 21, kColKEmpty, kColKFull, kColSEmpty, kColSFull };
+
+template <int D>
+__global__ void __launch_bounds__(kColThreads, 1)
+colsum_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUtensorMap tmk, const ColsumParams p) {
+  using L = ColsumSmem<D>;
+  constexpr int NPANEL = D / 64;
+  constexpr int KPANEL_BYTES = 128 * 128;
+  extern __shared__ __align__(1024) uint8_t smem[];
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int range = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+  const int kt0 = range * p.tiles_per_range;
+  const int ntile = min(p.NKT, kt0 + p.tiles_per_range) - kt0;
+  const int item = (b * p.H + h) * p.n_range + range;
+  const int W = p.W, NCH = p.NCH;
+  const int q_chunk_bytes = W * D * 2, q_panel_bytes = W * 128;
+  if (ntile <= 0) return;
+  if ((smem_u32(smem) & 1023u) != 0u) {
+    if (tid == 0) report_status(p.status, AVSA_ERR_CUDA, kWhereSmemAlign, item, 0);
+    return;
+  }
+  const int bars_off = L::kQ + NCH * q_chunk_bytes;
+  const uint32_t bar0 = smem_u32(smem + bars_off);
+  auto BAR = [&](int i) { return bar0 + static_cast<uint32_t>(i) * 8u; };
+  constexpr int Q_FULL = 0, K_FULL = 1, K_EMPTY = 1 + kColStages, S_FULL = 1 + 2 * kColStages, S_EMPTY = S_FULL + 2;
+  float* lse2 = reinterpret_cast<float*>(smem + bars_off + L::kBarBytes);
+  volatile uint32_t* misc = reinterpret_cast<volatile uint32_t*>(smem + bars_off + L::kBarBytes + 512 * 4);
+
+  if (tid == 0) {
+    mbar_init(BAR(Q_FULL), 1);
+    for (int s = 0; s < kColStages; s++) {
+      mbar_init(BAR(K_FULL + s), 1);
+      mbar_init(BAR(K_EMPTY + s), 1);
+    }
+    for (int g = 0; g < 2; g++) {
+      mbar_init(BAR(S_FULL + g), 1);
+      mbar_init(BAR(S_EMPTY + g), 128);
+    }
+    misc[1] = 0u;
+    fence_mbar_init();
+    prefetch_tmap(&tmq);
+    prefetch_tmap(&tmk);
+  }
+  for (int j = tid; j < NCH * W; j += kColThreads)
+    lse2[j] = (j < p.Nq) ? p.lse[(static_cast<int64_t>(b) * p.H + h) * p.Nq + j] * 1.4426950408889634f : INFINITY;
+  if (warp == 2) {
+    tmem_alloc(smem_u32(const_cast<uint32_t*>(misc)), 512);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = misc[0];
+
+  auto wait_or_abort = [&](int bar, uint32_t parity, int where, int aux) -> bool {
+    if (misc[1] != 0u) return false;
+    if (mbar_wait(BAR(bar), parity)) return true;
+    report_status(p.status, AVSA_ERR_TIMEOUT, where, item, aux);
+    misc[1] = 1u;
+    return false;
+  };
+
+  const int n_units = ntile * NCH;
+  if (warp == 0) {
+    if (lane == 0) {
+      mbar_expect_tx(BAR(Q_FULL), NCH * q_chunk_bytes);
+      for (int ch = 0; ch < NCH; ch++)
+        for (int pn = 0; pn < NPANEL; pn++)
+          tma_load_4d(smem_u32(smem + L::kQ) + ch * q_chunk_bytes + pn * q_panel_bytes, &tmq, BAR(Q_FULL), pn * 64,
+                      ch * W, h, b);
+      bool ok = true;
+      for (int t = 0; t < ntile && ok; t++) {
+        const int s = t % kColStages, f = t / kColStages;
+        if (f > 0) ok = wait_or_abort(K_EMPTY + s, (f - 1) & 1, kColKEmpty, t);
+        if (!ok) break;
+        mbar_expect_tx(BAR(K_FULL + s), L::kKTile);
+        for (int pn = 0; pn < NPANEL; pn++)
+          tma_load_4d(smem_u32(smem + L::kK) + s * L::kKTile + pn * KPANEL_BYTES, &tmk, BAR(K_FULL + s), pn * 64,
+                      (kt0 + t) * 128, h, b);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      const uint32_t idesc = make_idesc_bf16(128, W, 0, 0);
+      bool ok = wait_or_abort(Q_FULL, 0, kColQFull, 0);
+      for (int t = 0; t < ntile && ok; t++) {
+        const int s = t % kColStages, f = t / kColStages;
+        ok = wait_or_abort(K_FULL + s, f & 1, kColKFull, t);
+        if (!ok) break;
+        const uint32_t k_addr = smem_u32(smem + L::kK) + s * L::kKTile;
+        for (int ch = 0; ch < NCH && ok; ch++) {
+          const int u = t * NCH + ch, g = u & 1, i = u >> 1;
+          if (i > 0) ok = wait_or_abort(S_EMPTY + g, (i - 1) & 1, kColSEmpty, u);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t q_addr = smem_u32(smem + L::kQ) + ch * q_chunk_bytes;
+#pragma unroll
+          for (int ks = 0; ks < D / 16; ks++) {
+            const uint64_t ad = make_sdesc(k_addr + (ks >> 2) * KPANEL_BYTES + (ks & 3) * 32, 16, 1024);
+            const uint64_t bd = make_sdesc(q_addr + (ks >> 2) * q_panel_bytes + (ks & 3) * 32, 16, 1024);
+            umma_ss(tmem + g * 256, ad, bd, idesc, ks > 0 ? 1u : 0u);
+          }
+          umma_commit(BAR(S_FULL + g));
+        }
+        if (ok) umma_commit(BAR(K_EMPTY + s));
+      }
+    }
+  } else if (warp >= 4) {
+    const int g = (warp - 4) >> 2;
+    const int row = ((warp & 3) << 5) + lane;
+    const uint32_t lane_off = static_cast<uint32_t>((warp & 3) * 32) << 16;
+    bool ok = true;
+    for (int u = g; u < n_units && ok; u += 2) {
+      const int i = u >> 1, t = u / NCH, ch = u % NCH;
+      ok = wait_or_abort(S_FULL + g, i & 1, kColSFull, u);
+      if (!ok) break;
+      tc_fence_after();
+      const float* l2 = lse2 + ch * W;
+      float sum0 = 0.f, sum1 = 0.f;
+      const uint32_t base = tmem + g * 256 + lane_off;
+      int c = 0;
+      for (; c + 32 <= W; c += 32) {
+        uint32_t s[32];
+        tmem_ld32(base + c, s);
+        tmem_wait_ld();
+#pragma unroll
+        for (int j = 0; j < 32; j += 4) {
+          const float4 lv = *reinterpret_cast<const float4*>(l2 + c + j);
+          sum0 += fast_exp2(fmaf(__uint_as_float(s[j]), p.scale_log2, -lv.x));
+          sum1 += fast_exp2(fmaf(__uint_as_float(s[j + 1]), p.scale_log2, -lv.y));
+          sum0 += fast_exp2(fmaf(__uint_as_float(s[j + 2]), p.scale_log2, -lv.z));
+          sum1 += fast_exp2(fmaf(__uint_as_float(s[j + 3]), p.scale_log2, -lv.w));
+        }
+      }
+      if (c < W) {   // W is a multiple of 16
+        uint32_t s[16];
+        tmem_ld16(base + c, s);
+        tmem_wait_ld();
+#pragma unroll
+        for (int j = 0; j < 16; j += 4) {
+          const float4 lv = *reinterpret_cast<const float4*>(l2 + c + j);
+          sum0 += fast_exp2(fmaf(__uint_as_float(s[j]), p.scale_log2, -lv.x));
+          sum1 += fast_exp2(fmaf(__uint_as_float(s[j + 1]), p.scale_log2, -lv.y));
+          sum0 += fast_exp2(fmaf(__uint_as_float(s[j + 2]), p.scale_log2, -lv.z));
+          sum1 += fast_exp2(fmaf(__uint_as_float(s[j + 3]), p.scale_log2, -lv.w));
+        }
+      }
+      tc_fence_before();
+      mbar_arrive(BAR(S_EMPTY + g));
+      const int key = (kt0 + t) * 128 + row;
+      if (key < p.Nk)
+        p.partial[(static_cast<int64_t>(ch) * gridDim.z * p.H + static_cast<int64_t>(b) * p.H + h) * p.Nk + key] =
+            sum0 + sum1;
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 2) tmem_dealloc(tmem, 512);
+}
+
+// scores[b,i] = beta * scores[b,i] + gamma * sum_h sum_ch partial[ch][b,h,i], heads in ascending order
+__global__ void __launch_bounds__(256) head_sum_kernel(const float* __restrict__ partial, int NCH, int B, int H,
+                                                       int Nk, float beta, float gamma, float* __restrict__ scores) {
+  const int64_t idx = static_cast<int64_t>(blockIdx.x) * 256 + threadIdx.x;
+  if (idx >= static_cast<int64_t>(B) * Nk) return;
+  const int b = static_cast<int>(idx / Nk), i = static_cast<int>(idx % Nk);
+  float acc = 0.f;
+  for (int h = 0; h < H; h++)
+    for (int ch = 0; ch < NCH; ch++)
+      acc += partial[(static_cast<int64_t>(ch) * B * H + static_cast<int64_t>(b) * H + h) * Nk + i];
+  float out = gamma * acc;
+  if (beta != 0.f) out = fmaf(beta, scores[idx], out);
+  scores[idx] = out;
+}
+
+struct CrossPlan {
+  int blk, NQT, NKB, n_split, tps;           // pass 1 (key tiles of blk)
+  int NKT, NCH, W, n_range, tpr;             // pass 2 (key tiles of 128)
+  size_t off_part_o, off_part_lse, off_lse, off_partial, total;
+};
+
+static CrossPlan make_cross_plan(int B, int H, int Nq, int Nk, int d) {
+  CrossPlan c;
+  c.blk = d;   // (blk, d) = (128,128) or (64,64)
+  c.NQT = (Nq + c.blk - 1) / c.blk;
+  c.NKB = (Nk + c.blk - 1) / c.blk;
+  const int target = 296;   // about two CTAs per SM's worth of work items
+  int want_split = (target + B * H * c.NQT - 1) / (B * H * c.NQT);
+  if (want_split < 1) want_split = 1;
+  if (want_split > c.NKB) want_split = c.NKB;
+  c.tps = (c.NKB + want_split - 1) / want_split;
+  c.n_split = (c.NKB + c.tps - 1) / c.tps;
+  c.NKT = (Nk + 127) / 128;
+  c.NCH = Nq > 256 ? 2 : 1;
+  c.W = (((Nq + c.NCH - 1) / c.NCH) + 15) / 16 * 16;
+  int want_range = (target + B * H - 1) / (B * H);
+  if (want_range < 1) want_range = 1;
+  if (want_range > c.NKT) want_range = c.NKT;
+  c.tpr = (c.NKT + want_range - 1) / want_range;
+  c.n_range = (c.NKT + c.tpr - 1) / c.tpr;
+  size_t off = kStatusBytes;
+  const size_t items = static_cast<size_t>(B) * H * c.NQT * c.n_split;
+  c.off_part_o = off; off += align_up(items * c.blk * d * sizeof(float), 256);
+  c.off_part_lse = off; off += align_up(items * c.blk * sizeof(float), 256);
+  c.off_lse = off; off += align_up(static_cast<size_t>(B) * H * Nq * sizeof(float), 256);
+  c.off_partial = off; off += align_up(static_cast<size_t>(c.NCH) * B * H * Nk * sizeof(float), 256);
+  c.total = off;
+  return c;
+}
+
+template <int BLK, int D>
+static int run_cross(int B, int H, int Nq, int Nk, const avsa_bf16_4d& q, const avsa_bf16_4d& k, const avsa_bf16_4d& v,
+                     void* o, float* lse_out, float* scores, float beta, float gamma, float scale, uint8_t* ws,
+                     const CrossPlan& c, cudaStream_t st) {
+  StatusRecord* status = reinterpret_cast<StatusRecord*>(ws);
+  float* part_o = reinterpret_cast<float*>(ws + c.off_part_o);
+  float* part_lse = reinterpret_cast<float*>(ws + c.off_part_lse);
+  float* lse = lse_out != nullptr ? lse_out : reinterpret_cast<float*>(ws + c.off_lse);
+  float* partial = reinterpret_cast<float*>(ws + c.off_partial);
+  clear_status_kernel<<<1, 1, 0, st>>>(status);
+  // ---- pass 1
+  {
+    using L = AttnSmem<BLK, D>;
+    CUtensorMap tq, tk, tv;
+    if (!encode_bf16_tile_map(&tq, q.ptr, B, H, Nq, D, q.stride_b, q.stride_h, q.stride_n, BLK)) return AVSA_ERR_CUDA;
+    if (!encode_bf16_tile_map(&tk, k.ptr, B, H, Nk, D, k.stride_b, k.stride_h, k.stride_n, BLK)) return AVSA_ERR_CUDA;
+    if (!encode_bf16_tile_map(&tv, v.ptr, B, H, Nk, D, v.stride_b, v.stride_h, v.stride_n, BLK)) return AVSA_ERR_CUDA;
+    if (cudaFuncSetAttribute(attn_fwd_kernel<BLK, D, MODE_RANGE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             L::kTotal) != cudaSuccess)
+      return AVSA_ERR_CUDA;
+    AttnParams prm = {};
+    prm.part_o = part_o;
+    prm.part_lse2 = part_lse;
+    prm.n_split = c.n_split;
+    prm.tiles_per_split = c.tps;
+    prm.status = status;
+    prm.H = H;
+    prm.Nq = Nq;
+    prm.NQT = c.NQT;
+    prm.Nk = Nk;
+    prm.NKB = c.NKB;
+    prm.scale_log2 = scale * 1.4426950408889634f;
+    dim3 grid(c.NQT * c.n_split, H, B);
+    attn_fwd_kernel<BLK, D, MODE_RANGE><<<grid, kAttnThreads, L::kTotal, st>>>(tq, tk, tv, tq, prm);
+    const int total_rows = B * H * Nq;
+    constexpr int RPB = 128 / (D / 4);
+    merge_splits_kernel<BLK, D><<<(total_rows + RPB - 1) / RPB, 128, 0, st>>>(
+        part_o, part_lse, c.n_split, c.NQT, Nq, H, total_rows, static_cast<__nv_bfloat16*>(o), q.stride_b, q.stride_h,
+        q.stride_n, lse);
+  }
+  // ---- pass 2
+  if (scores != nullptr) {
+    using L = ColsumSmem<D>;
+    CUtensorMap tq, tk;
+    if (!encode_bf16_tile_map(&tq, q.ptr, B, H, Nq, D, q.stride_b, q.stride_h, q.stride_n, c.W)) return AVSA_ERR_CUDA;
+    if (!encode_bf16_tile_map(&tk, k.ptr, B, H, Nk, D, k.stride_b, k.stride_h, k.stride_n, 128)) return AVSA_ERR_CUDA;
+    const int smem = L::total(c.NCH, c.W);
+    if (cudaFuncSetAttribute(colsum_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
+      return AVSA_ERR_CUDA;
+    ColsumParams cp;
+    cp.lse = lse;
+    cp.partial = partial;
+    cp.status = status;
+    cp.H = H;
+    cp.Nq = Nq;
+    cp.Nk = Nk;
+    cp.NKT = c.NKT;
+    cp.NCH = c.NCH;
+    cp.W = c.W;
+    cp.n_range = c.n_range;
+    cp.tiles_per_range = c.tpr;
+    cp.scale_log2 = scale * 1.4426950408889634f;
+    dim3 grid(c.n_range, H, B);
+    colsum_kernel<D><<<grid, kColThreads, smem, st>>>(tq, tk, cp);
+    const int64_t n = static_cast<int64_t>(B) * Nk;
+    head_sum_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, st>>>(partial, c.NCH, B, H, Nk, beta, gamma,
+                                                                           scores);
+  }
+  return cudaGetLastError() == cudaSuccess ? AVSA_OK : AVSA_ERR_CUDA;
+}
+
+}  // namespace avsa
+
+using namespace avsa;
+
+extern "C" size_t avsa_cross_attn_scores_workspace_bytes(int B, int H, int Nq, int Nk, int d) {
+  if (B <= 0 || H <= 0 || Nq <= 0 || Nk <= 0 || (d != 64 && d != 128)) return 0;
+  return make_cross_plan(B, H, Nq, Nk, d).total;
+}
+
+extern "C" int avsa_cross_attn_scores(int B, int H, int Nq, int Nk, int d, avsa_bf16_4d q, avsa_bf16_4d k,
+                                      avsa_bf16_4d v, void* o_bf16, float* lse, float* scores, float score_beta,
+                                      float score_gamma, float softmax_scale, void* ws, size_t ws_bytes,
+                                      void* stream) {
+  if (B <= 0 || H <= 0 || Nq <= 0 || Nk <= 0) return AVSA_ERR_INVALID_ARG;
+  if (d != 64 && d != 128) return AVSA_ERR_UNSUPPORTED;
+  if (Nq > 512 || H > 65535 || B > 65535) return AVSA_ERR_UNSUPPORTED;
+  if (!tensor_ok(q, B, H) || !tensor_ok(k, B, H) || !tensor_ok(v, B, H)) return AVSA_ERR_INVALID_ARG;
+  if (o_bf16 != nullptr && !aligned16(o_bf16)) return AVSA_ERR_INVALID_ARG;
+  if (softmax_scale < 0.f || softmax_scale != softmax_scale) return AVSA_ERR_INVALID_ARG;
+  const CrossPlan c = make_cross_plan(B, H, Nq, Nk, d);
+  if (ws == nullptr || ws_bytes < c.total) return AVSA_ERR_WORKSPACE;
+  if (!device_is_sm100()) return AVSA_ERR_UNSUPPORTED;
+  const float scale = softmax_scale != 0.f ? softmax_scale : 1.0f / sqrtf(static_cast<float>(d));
+  uint8_t* base = static_cast<uint8_t*>(ws);
+  if (d == 128)
+    return run_cross<128, 128>(B, H, Nq, Nk, q, k, v, o_bf16, lse, scores, score_beta, score_gamma, scale, base, c,
+                               as_stream(stream));
+  return run_cross<64, 64>(B, H, Nq, Nk, q, k, v, o_bf16, lse, scores, score_beta, score_gamma, scale, base, c,
+                           as_stream(stream));
+}

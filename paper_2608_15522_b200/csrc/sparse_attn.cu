@@ -1,0 +1,59 @@
+// avsa_sparse_self_attn: block-sparse video self-attention under the protected block mask
+// (Eq. 10 / Eq. 11; Eq. 5 when every list is full).  Host side: argument checks, tensor maps, launch.
+#include "attn_kernel.cuh"
+
+namespace avsa {
+
+template <int BLK, int D>
+static int launch_sparse_attn(int B, int H, int N, const avsa_bf16_4d& q, const avsa_bf16_4d& k,
+                              const avsa_bf16_4d& v, void* o, const AttnParams& prm, cudaStream_t st) {
+  using L = AttnSmem<BLK, D>;
+  CUtensorMap tq, tk, tv, to;
+  if (!encode_bf16_tile_map(&tq, q.ptr, B, H, N, D, q.stride_b, q.stride_h, q.stride_n, BLK)) return AVSA_ERR_CUDA;
+  if (!encode_bf16_tile_map(&tk, k.ptr, B, H, N, D, k.stride_b, k.stride_h, k.stride_n, BLK)) return AVSA_ERR_CUDA;
+  if (!encode_bf16_tile_map(&tv, v.ptr, B, H, N, D, v.stride_b, v.stride_h, v.stride_n, BLK)) return AVSA_ERR_CUDA;
+  if (!encode_bf16_tile_map(&to, o, B, H, N, D, q.stride_b, q.stride_h, q.stride_n, BLK)) return AVSA_ERR_CUDA;
+  if (cudaFuncSetAttribute(attn_fwd_kernel<BLK, D, MODE_LIST>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           L::kTotal) != cudaSuccess)
+    return AVSA_ERR_CUDA;
+  dim3 grid(prm.NQT, H, B);
+  attn_fwd_kernel<BLK, D, MODE_LIST><<<grid, kAttnThreads, L::kTotal, st>>>(tq, tk, tv, to, prm);
+  return cudaGetLastError() == cudaSuccess ? AVSA_OK : AVSA_ERR_CUDA;
+}
+
+}  // namespace avsa
+
+using namespace avsa;
+
+extern "C" size_t avsa_sparse_self_attn_workspace_bytes(int B, int H, int N, int d, int blk) {
+  if (B <= 0 || H <= 0 || N <= 0 || d <= 0 || blk <= 0) return 0;
+  return kStatusBytes;
+}
+
+extern "C" int avsa_sparse_self_attn(int B, int H, int N, int d, int blk, avsa_bf16_4d q, avsa_bf16_4d k,
+                                     avsa_bf16_4d v, const int32_t* col_idx, const int32_t* col_cnt, void* o_bf16,
+                                     float* lse, float softmax_scale, void* ws, size_t ws_bytes, void* stream) {
+  if (B <= 0 || H <= 0 || N <= 0) return AVSA_ERR_INVALID_ARG;
+  if (!((blk == 128 && d == 128) || (blk == 64 && d == 64))) return AVSA_ERR_UNSUPPORTED;
+  if (H > 65535 || B > 65535) return AVSA_ERR_UNSUPPORTED;
+  if (!tensor_ok(q, B, H) || !tensor_ok(k, B, H) || !tensor_ok(v, B, H)) return AVSA_ERR_INVALID_ARG;
+  if (col_idx == nullptr || col_cnt == nullptr || o_bf16 == nullptr || !aligned16(o_bf16)) return AVSA_ERR_INVALID_ARG;
+  if (softmax_scale < 0.f || softmax_scale != softmax_scale) return AVSA_ERR_INVALID_ARG;
+  if (ws == nullptr || ws_bytes < kStatusBytes) return AVSA_ERR_WORKSPACE;
+  if (!device_is_sm100()) return AVSA_ERR_UNSUPPORTED;
+  cudaStream_t st = as_stream(stream);
+  AttnParams prm = {};
+  prm.col_idx = col_idx;
+  prm.col_cnt = col_cnt;
+  prm.lse = lse;
+  prm.status = static_cast<StatusRecord*>(ws);
+  prm.H = H;
+  prm.Nq = N;
+  prm.Nk = N;
+  prm.NQT = prm.NKB = (N + blk - 1) / blk;
+  const float scale = softmax_scale != 0.f ? softmax_scale : 1.0f / sqrtf(static_cast<float>(d));
+  prm.scale_log2 = scale * 1.4426950408889634f;
+  clear_status_kernel<<<1, 1, 0, st>>>(prm.status);
+  if (d == 128) return launch_sparse_attn<128, 128>(B, H, N, q, k, v, o_bf16, prm, st);
+  return launch_sparse_attn<64, 64>(B, H, N, q, k, v, o_bf16, prm, st);
+}

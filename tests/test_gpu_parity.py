@@ -1,0 +1,306 @@
+"""GPU parity: every call of the C ABI against the fp64 CPU oracle on the same seeded inputs.
+
+Bars: integer outputs (flags, lists, counts) bit-exact given the same fp32 score tensors;
+floating-point outputs within max-abs 1e-2 and relative-L2 5e-3 of the oracle (bf16 inputs, fp32
+accumulation, bf16 probabilities in the P.V product).
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import avsa_oracle as orc
+from paper_2608_15522_b200 import binding as av
+from paper_2608_15522_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+MAX_ABS = 1e-2
+REL_L2 = 5e-3
+
+
+def _np64(x):
+    return x.detach().double().cpu().numpy()
+
+
+def _close(got, want, what):
+    got = np.asarray(got, np.float64)
+    want = np.asarray(want, np.float64)
+    # max-abs 1e-2 for values up to magnitude 1; beyond that the bound scales with the value, because
+    # the bf16 output grid itself is coarser than 1e-2 there (half-spacing 2^-7 at |x| in [2,4))
+    err = (np.abs(got - want) / np.maximum(1.0, np.abs(want))).max()
+    rel = np.linalg.norm((got - want).ravel()) / max(np.linalg.norm(want.ravel()), 1e-30)
+    assert np.isfinite(got).all(), f"{what}: non-finite values"
+    assert err <= MAX_ABS, f"{what}: max-abs (scaled) {err:.3e} > {MAX_ABS}"
+    assert rel <= REL_L2, f"{what}: rel-L2 {rel:.3e} > {REL_L2}"
+
+
+def _status_ok(ws):
+    code, detail = av.avsa_read_status(ws)
+    assert code == av.AVSA_OK, f"device status {code} {av.status_string(code)} detail {detail}"
+
+
+def _oracle_mask(w, q, k, scores64, n_protect, k_keep, flags=av.AVSA_PROTECT_ROWS):
+    """Oracle block scores (rounded to fp32, the tensor both sides select from) and its lists."""
+    bs32 = orc.block_scores(_np64(q), _np64(k), w.blk).astype(np.float32)
+    s32 = scores64.astype(np.float32)
+    idx, cnt, ptok, pblk = orc.build_block_mask(bs32, s32, n_protect, k_keep, w.blk, w.n_video,
+                                                bool(flags & av.AVSA_PROTECT_ROWS), bool(flags & av.AVSA_PROTECT_COLS))
+    return bs32, s32, idx, cnt, ptok, pblk
+
+
+def _oracle_scores(w, seed):
+    qa, kc, vc = wl.make_cross_qkv(w, seed)
+    o, lse, A = orc.cross_attention(_np64(qa), _np64(kc), _np64(vc))
+    s = orc.column_scores(A, gamma=1.0 / (w.H * w.n_audio))
+    return (qa, kc, vc), o, lse, s
+
+
+# ------------------------------------------------------------------------------------------- mask
+@pytest.mark.parametrize("name,flags", [("tiny", 1), ("small128", 1), ("medium128", 1), ("medium128", 3)])
+def test_mask_lists_bit_exact_given_oracle_scores(name, flags):
+    w = wl.WORKLOADS[name]
+    q, k, _ = wl.make_self_qkv(w, 0)
+    _, _, _, s64 = _oracle_scores(w, 0)
+    n_protect = orc.ceil_pct(w.protect_pct, w.n_video)
+    k_keep = max(1, orc.ceil_pct(w.keep_pct, w.n_blocks))
+    assert n_protect == av.avsa_count_from_percent(w.protect_pct, w.n_video)
+    assert k_keep == max(1, av.avsa_count_from_percent(w.keep_pct, w.n_blocks))
+    bs32, s32, idx, cnt, ptok, pblk = _oracle_mask(w, q, k, s64, n_protect, k_keep, flags)
+    out = av.avsa_build_block_mask(None, None, torch.from_numpy(s32).cuda(), n_protect, k_keep, w.blk,
+                                   flags=flags | av.AVSA_USE_GIVEN_BLOCK_SCORES,
+                                   block_scores=torch.from_numpy(bs32).cuda(), shape=(w.B, w.H, w.n_video, w.d))
+    _status_ok(out["ws"])
+    assert np.array_equal(out["prot_tok"].cpu().numpy(), ptok)
+    assert np.array_equal(out["prot_blk"].cpu().numpy(), pblk)
+    assert np.array_equal(out["col_cnt"].cpu().numpy(), cnt)
+    assert np.array_equal(out["col_idx"].cpu().numpy(), idx)
+
+
+def test_mask_ties_nan_and_signed_zero_bit_exact():
+    B, H, N, d, blk = 2, 2, 64 * 37 + 5, 64, 64
+    NB = (N + blk - 1) // blk
+    rng = np.random.default_rng(3)
+    bs = rng.integers(-2, 3, size=(B, H, NB, NB)).astype(np.float32)          # heavy ties
+    bs[0, 0, 1, :] = 0.0
+    bs[0, 0, 2, ::2] = -0.0
+    bs[0, 1, 3, 5] = np.nan
+    bs[1, 0, 4, :] = np.nan
+    bs[1, 1, 5, 7] = np.inf
+    bs[1, 1, 5, 9] = -np.inf
+    s = rng.integers(0, 4, size=(B, N)).astype(np.float32)
+    s[0, 10] = np.nan
+    s[1, ::3] = -0.0
+    for n_protect, k_keep in ((0, 1), (7, 5), (200, NB), (N, 3), (1, NB - 1)):
+        idx, cnt, ptok, pblk = orc.build_block_mask(bs, s, n_protect, k_keep, blk, N)
+        out = av.avsa_build_block_mask(None, None, torch.from_numpy(s).cuda(), n_protect, k_keep, blk,
+                                       flags=av.AVSA_PROTECT_ROWS | av.AVSA_USE_GIVEN_BLOCK_SCORES,
+                                       block_scores=torch.from_numpy(bs).cuda(), shape=(B, H, N, d))
+        _status_ok(out["ws"])
+        assert np.array_equal(out["prot_tok"].cpu().numpy(), ptok), (n_protect, k_keep)
+        assert np.array_equal(out["prot_blk"].cpu().numpy(), pblk), (n_protect, k_keep)
+        assert np.array_equal(out["col_cnt"].cpu().numpy(), cnt), (n_protect, k_keep)
+        assert np.array_equal(out["col_idx"].cpu().numpy(), idx), (n_protect, k_keep)
+
+
+@pytest.mark.parametrize("name", ["tiny", "small128", "medium128"])
+def test_block_scores_and_selection_from_pooled_qk(name):
+    w = wl.WORKLOADS[name]
+    q, k, _ = wl.make_self_qkv(w, 1)
+    _, _, _, s64 = _oracle_scores(w, 1)
+    n_protect = orc.ceil_pct(w.protect_pct, w.n_video)
+    k_keep = max(1, orc.ceil_pct(w.keep_pct, w.n_blocks))
+    s32 = s64.astype(np.float32)
+    out = av.avsa_build_block_mask(q.cuda(), k.cuda(), torch.from_numpy(s32).cuda(), n_protect, k_keep, w.blk)
+    _status_ok(out["ws"])
+    want = orc.block_scores(_np64(q), _np64(k), w.blk)
+    got = out["block_scores"].cpu().numpy()
+    assert np.abs(got - want).max() <= 1e-4 * max(1.0, np.abs(want).max())
+    # the lists are exactly the oracle's when it selects from the very tensor the GPU produced
+    idx, cnt, ptok, pblk = orc.build_block_mask(got, s32, n_protect, k_keep, w.blk, w.n_video)
+    assert np.array_equal(out["col_idx"].cpu().numpy(), idx)
+    assert np.array_equal(out["col_cnt"].cpu().numpy(), cnt)
+    assert np.array_equal(out["prot_tok"].cpu().numpy(), ptok)
+    # and a valid top-k of the oracle's own fp64 scores up to the fp32 rounding of the scores
+    gidx, gcnt = out["col_idx"].cpu().numpy(), out["col_cnt"].cpu().numpy()
+    tol = 2e-4 * max(1.0, np.abs(want).max())
+    for b in range(w.B):
+        for h in range(w.H):
+            for i in range(w.n_blocks):
+                if pblk[b, i] or k_keep >= w.n_blocks:
+                    continue
+                kept = gidx[b, h, i, : gcnt[b, h, i]]
+                rest = np.setdiff1d(np.arange(w.n_blocks), kept)
+                assert want[b, h, i, kept].min() >= want[b, h, i, rest].max() - tol
+
+
+# ------------------------------------------------------------------------------------------- sparse attention
+def _run_sparse_case(w, seed, idx, cnt, want_lse=True):
+    q, k, v = wl.make_self_qkv(w, seed)
+    o, lse, ws = av.avsa_sparse_self_attn(q.cuda(), k.cuda(), v.cuda(), torch.from_numpy(idx).cuda(),
+                                          torch.from_numpy(cnt).cuda(), w.blk, want_lse=want_lse)
+    _status_ok(ws)
+    want_o, want_l = orc.masked_attention(_np64(q), _np64(k), _np64(v), idx, cnt, w.blk)
+    _close(_np64(o), want_o, f"{w.name} O")
+    if want_lse:
+        _close(_np64(lse), want_l, f"{w.name} lse")
+    return _np64(o), want_o
+
+
+@pytest.mark.parametrize("name", ["tiny", "small128", "medium128"])
+def test_sparse_attention_matches_oracle_under_protected_mask(name):
+    w = wl.WORKLOADS[name]
+    q, k, _ = wl.make_self_qkv(w, 0)
+    _, _, _, s64 = _oracle_scores(w, 0)
+    n_protect = orc.ceil_pct(w.protect_pct, w.n_video)
+    k_keep = max(1, orc.ceil_pct(w.keep_pct, w.n_blocks))
+    _, _, idx, cnt, _, pblk = _oracle_mask(w, q, k, s64, n_protect, k_keep)
+    assert 0 < pblk.sum() < pblk.size or name == "small128"
+    _run_sparse_case(w, 0, idx, cnt)
+
+
+@pytest.mark.parametrize("name", ["tiny", "small128", "medium128"])
+def test_sparse_attention_keep_all_is_dense(name):
+    w = wl.WORKLOADS[name]
+    NB = w.n_blocks
+    idx = np.broadcast_to(np.arange(NB, dtype=np.int32), (w.B, w.H, NB, NB)).copy()
+    cnt = np.full((w.B, w.H, NB), NB, np.int32)
+    got, _ = _run_sparse_case(w, 2, idx, cnt)
+    q, k, v = wl.make_self_qkv(w, 2)
+    dense, _ = orc.dense_attention(_np64(q), _np64(k), _np64(v))
+    _close(got, dense, f"{name} keep-all vs dense")
+
+
+def test_sparse_attention_single_and_odd_counts():
+    """Lists of 1, 2 and 3 entries, and the last (ragged) key block alone."""
+    w = wl.WORKLOADS["medium128"]
+    NB = w.n_blocks
+    idx = np.full((w.B, w.H, NB, NB), -1, np.int32)
+    cnt = np.zeros((w.B, w.H, NB), np.int32)
+    rng = np.random.default_rng(5)
+    for b in range(w.B):
+        for h in range(w.H):
+            for i in range(NB):
+                c = 1 + (i % 3)
+                cols = np.sort(rng.choice(NB, size=c, replace=False))
+                if i == 4:
+                    cols = np.array([NB - 1])
+                idx[b, h, i, :c] = cols
+                cnt[b, h, i] = len(cols)
+    _run_sparse_case(w, 3, idx, cnt)
+
+
+def test_sparse_attention_strided_bnhd_layout():
+    w = wl.WORKLOADS["small128"]
+    q, k, v = wl.make_self_qkv(w, 4)
+    NB = w.n_blocks
+    idx = np.broadcast_to(np.arange(NB, dtype=np.int32), (w.B, w.H, NB, NB)).copy()
+    cnt = np.full((w.B, w.H, NB), NB, np.int32)
+    # storage [B,N,H,d], viewed as [B,H,N,d]
+    qs, ks, vs = (t.cuda().permute(0, 2, 1, 3).contiguous().permute(0, 2, 1, 3) for t in (q, k, v))
+    assert not qs.is_contiguous()
+    o, _, ws = av.avsa_sparse_self_attn(qs, ks, vs, torch.from_numpy(idx).cuda(), torch.from_numpy(cnt).cuda(), w.blk)
+    _status_ok(ws)
+    assert o.stride() == qs.stride()
+    want, _ = orc.dense_attention(_np64(q), _np64(k), _np64(v))
+    _close(_np64(o), want, "strided O")
+
+
+def test_sparse_attention_rejects_malformed_lists_without_touching_memory():
+    w = wl.WORKLOADS["small128"]
+    q, k, v = (t.cuda() for t in wl.make_self_qkv(w, 0))
+    NB = w.n_blocks
+    for bad in ([0, 0], [2, 1], [0, NB], [-1, 1]):
+        idx = np.broadcast_to(np.arange(NB, dtype=np.int32), (w.B, w.H, NB, NB)).copy()
+        cnt = np.full((w.B, w.H, NB), NB, np.int32)
+        idx[0, 1, 2, :2] = bad
+        cnt[0, 1, 2] = 2
+        o, _, ws = av.avsa_sparse_self_attn(q, k, v, torch.from_numpy(idx).cuda(), torch.from_numpy(cnt).cuda(), w.blk)
+        code, detail = av.avsa_read_status(ws)
+        assert code == av.AVSA_ERR_BAD_MASK
+        assert detail[1] == (0 * w.H + 1) * NB + 2
+    cnt = np.zeros((w.B, w.H, NB), np.int32)
+    o, _, ws = av.avsa_sparse_self_attn(q, k, v, torch.from_numpy(idx).cuda(), torch.from_numpy(cnt).cuda(), w.blk)
+    assert av.avsa_read_status(ws)[0] == av.AVSA_ERR_BAD_MASK
+
+
+# ------------------------------------------------------------------------------------------- cross attention
+@pytest.mark.parametrize("name", ["tiny", "small128", "medium128"])
+def test_cross_attention_outputs_and_scores(name):
+    w = wl.WORKLOADS[name]
+    (qa, kc, vc), want_o, want_lse, want_s = _oracle_scores(w, 0)
+    gamma = 1.0 / (w.H * w.n_audio)
+    o, lse, s, ws = av.avsa_cross_attn_scores(qa.cuda(), kc.cuda(), vc.cuda(), score_gamma=gamma)
+    _status_ok(ws)
+    _close(_np64(o), want_o, f"{name} cross O")
+    _close(_np64(lse), want_lse, f"{name} cross lse")
+    got_s = _np64(s)
+    assert abs(got_s.sum() - w.B) < 2e-3 * w.B                          # rows of Eq. 1 sum to one
+    rel = np.linalg.norm(got_s - want_s) / np.linalg.norm(want_s)
+    assert rel <= REL_L2 and np.abs(got_s - want_s).max() <= MAX_ABS
+    # running blend (Eq. 4) and bit-for-bit reproducibility
+    prev = torch.rand_like(s)
+    s2 = prev.clone()
+    av.avsa_cross_attn_scores(qa.cuda(), kc.cuda(), vc.cuda(), scores=s2, score_beta=0.25, score_gamma=0.75 * gamma)
+    torch.cuda.synchronize()
+    want2 = 0.25 * _np64(prev) + 0.75 * want_s
+    assert np.linalg.norm(_np64(s2) - want2) / np.linalg.norm(want2) <= REL_L2
+    _, _, s3, _ = av.avsa_cross_attn_scores(qa.cuda(), kc.cuda(), vc.cuda(), score_gamma=gamma)
+    assert torch.equal(s, s3)
+
+
+def test_cross_attention_long_query_axis_two_chunks():
+    """More than 256 queries: the column-sum pass splits the query axis in two."""
+    w = wl.Workload("x", 1, 2, 128, 2, 9, 17, 300, 128, 50, 10, 1.0, ((0, 1, 1, 3, 2, 4),))
+    (qa, kc, vc), want_o, want_lse, want_s = _oracle_scores(w, 7)
+    o, lse, s, ws = av.avsa_cross_attn_scores(qa.cuda(), kc.cuda(), vc.cuda(), score_gamma=1.0 / (w.H * w.n_audio))
+    _status_ok(ws)
+    _close(_np64(o), want_o, "cross O")
+    _close(_np64(lse), want_lse, "cross lse")
+    assert np.linalg.norm(_np64(s) - want_s) / np.linalg.norm(want_s) <= REL_L2
+
+
+# ------------------------------------------------------------------------------------------- whole path
+def test_whole_path_tiny_matches_oracle():
+    w = wl.WORKLOADS["tiny"]
+    qa, kc, vc = (t.cuda() for t in wl.make_cross_qkv(w, 0))
+    q, k, v = (t.cuda() for t in wl.make_self_qkv(w, 0))
+    n_protect = av.avsa_count_from_percent(w.protect_pct, w.n_video)
+    k_keep = av.avsa_count_from_percent(w.keep_pct, w.n_blocks)
+    assert (n_protect, k_keep) == (26, 2)
+    _, _, s, _ = av.avsa_cross_attn_scores(qa, kc, vc, score_gamma=1.0 / (w.H * w.n_audio))
+    m = av.avsa_build_block_mask(q, k, s, n_protect, k_keep, w.blk)
+    o, _, ws = av.avsa_sparse_self_attn(q, k, v, m["col_idx"], m["col_cnt"], w.blk)
+    _status_ok(ws)
+    # oracle end to end
+    _, _, A = orc.cross_attention(_np64(qa), _np64(kc), _np64(vc))
+    s64 = orc.column_scores(A, gamma=1.0 / (w.H * w.n_audio))
+    bs64 = orc.block_scores(_np64(q), _np64(k), w.blk)
+    idx, cnt, ptok, pblk = orc.build_block_mask(bs64, s64, n_protect, k_keep, w.blk, w.n_video)
+    region = wl.region_mask(w, "cpu").numpy()
+    assert (ptok[0].astype(bool) & region).sum() >= 24                    # the planted region is what gets protected
+    # the planted margin makes the selections agree exactly between fp32/bf16 GPU scores and fp64 oracle
+    assert np.array_equal(m["prot_blk"].cpu().numpy(), pblk)
+    assert np.array_equal(m["col_cnt"].cpu().numpy(), cnt)
+    assert np.array_equal(m["col_idx"].cpu().numpy(), idx)
+    want, _ = orc.masked_attention(_np64(q), _np64(k), _np64(v), idx, cnt, w.blk)
+    _close(_np64(o), want, "whole path O")
+
+
+def test_host_side_argument_errors():
+    w = wl.WORKLOADS["tiny"]
+    q, k, v = (t.cuda() for t in wl.make_self_qkv(w, 0))
+    NB = w.n_blocks
+    idx = torch.zeros((1, 2, NB, NB), dtype=torch.int32, device="cuda")
+    cnt = torch.ones((1, 2, NB), dtype=torch.int32, device="cuda")
+    with pytest.raises(av.AvsaError) as e:
+        av.avsa_sparse_self_attn(q, k, v, idx, cnt, 32)
+    assert e.value.status == av.AVSA_ERR_UNSUPPORTED
+    with pytest.raises(av.AvsaError) as e:
+        av.avsa_sparse_self_attn(q, k, v, idx, cnt, w.blk, ws=torch.empty(256, dtype=torch.uint8, device="cuda")[:8])
+    assert e.value.status == av.AVSA_ERR_WORKSPACE
+    with pytest.raises(av.AvsaError) as e:
+        av.avsa_build_block_mask(q, k, None, 3, 1, w.blk)
+    assert e.value.status == av.AVSA_ERR_INVALID_ARG
+    with pytest.raises(av.AvsaError) as e:
+        av.avsa_build_block_mask(q, k, None, 0, NB + 1, w.blk)
+    assert e.value.status == av.AVSA_ERR_INVALID_ARG
