@@ -1,0 +1,369 @@
+#!/usr/bin/env python
+"""Benchmark of the protected sparse video-attention layer-step on B200.
+
+One step = the whole hot path on one batch of synthetic input:
+  avsa_cross_attn_scores (Eq. 1-2)  ->  avsa_build_block_mask (Eq. 8-9)  ->  avsa_sparse_self_attn (Eq. 10)
+on the Ovi-class single-layer workload (24 heads, d 128, 32760 video tokens, 256 audio tokens, block 128,
+keep 25 %, protect 5 %).  Prints ONE JSON line (rank 0).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload ovi|ltx|mid|tiny] [--impl ours|reference]
+
+N > 1 runs one independent replica of the layer per GPU (weak scaling, no data-path collective); launch with
+torchrun.  ``--impl reference`` times the fp64 CPU oracle on the host cores on a bounded sample of the workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2608_15522_b200 import workloads as wl  # noqa: E402
+
+METRIC = "dense-equiv TFLOP/s of protected sparse video attn (layer-step: cross-attn scores + mask + sparse attn)"
+UNIT = "TFLOP/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the sparse attention kernel, from the ncu capture
+# summarised under profiles/ (None until a capture exists for that workload)
+NCU_TRAFFIC_BYTES = {}
+KERNELS_PER_STEP = 12   # cross: clear, pass 1, merge, pass 2, head sum; mask: clear, select, pool, scores, rows; attn: clear, attn
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return p, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+def dense_flops(w):
+    return 4.0 * w.B * w.H * float(w.n_video) ** 2 * w.d
+
+
+# ------------------------------------------------------------------------------------------------ clocks
+class ClockSampler:
+    """Samples SM clocks and throttle reasons of one GPU with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.lines:
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 8:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[4:8]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------------------------------------ CPU oracle arm
+def oracle_sample(w, q_blocks=4):
+    """Times the oracle on head 0 of the workload: Eq. 1-2 for one head, block scores for one head, the mask step
+    on those, and Eq. 10 for ``q_blocks`` query blocks at full key length.  Returns (seconds extrapolated to a
+    whole layer, description, measured seconds)."""
+    from oracle import avsa_oracle as orc
+    one = wl.Workload(w.name, 1, 1, w.d, w.frames, w.rows, w.cols, w.n_audio, w.blk, w.keep_pct, w.protect_pct,
+                      w.a_pos, w.regions)
+    q, k, v = (t.double().numpy() for t in wl.make_self_qkv(one, 0))
+    qa, kc, vc = (t.double().numpy() for t in wl.make_cross_qkv(one, 0))
+    NB = w.n_blocks
+    n_protect = orc.ceil_pct(w.protect_pct, w.n_video)
+    k_keep = max(1, orc.ceil_pct(w.keep_pct, NB))
+    t0 = time.perf_counter()
+    _, _, A = orc.cross_attention(qa, kc, vc)
+    s = orc.column_scores(A, gamma=1.0 / (w.n_audio))
+    del A
+    t1 = time.perf_counter()
+    bs = orc.block_scores(q, k, w.blk)
+    idx, cnt, _, pblk = orc.build_block_mask(bs.astype(np.float32), s.astype(np.float32), n_protect, k_keep, w.blk,
+                                             w.n_video)
+    t2 = time.perf_counter()
+    prot = [i for i in range(NB) if pblk[0, i]]
+    unprot = [i for i in range(NB) if not pblk[0, i]]
+    half = max(1, q_blocks // 2)
+    chosen = (prot[:half] + unprot[: q_blocks - len(prot[:half])])[:q_blocks] or [0]
+    pairs_sample = 0
+    for i in chosen:
+        lo, hi = i * w.blk, min((i + 1) * w.blk, w.n_video)
+        cols = [int(c) for c in idx[0, 0, i, : int(cnt[0, 0, i])]]
+        orc.masked_attention_rows(q[0, 0, lo:hi], k[0, 0], v[0, 0], cols, w.blk)
+        pairs_sample += len(cols)
+    t3 = time.perf_counter()
+    pairs_head = int(cnt[0, 0].sum())
+    per_layer = w.B * w.H * ((t1 - t0) + (t2 - t1) + (t3 - t2) * pairs_head / max(pairs_sample, 1))
+    desc = (f"head 0 of {w.name}: Eq.1-2 oracle ({t1 - t0:.2f}s) + block scores and mask ({t2 - t1:.2f}s) + Eq.10 oracle "
+            f"on {len(chosen)} query blocks x full key lists ({t3 - t2:.2f}s); layer time extrapolated by heads and "
+            f"by executed block pairs ({pairs_sample} of {pairs_head} per head)")
+    return per_layer, desc, t3 - t0
+
+
+def run_reference(args, w):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cores = len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else os.cpu_count()
+    for _ in range(min(args.warmup, 1)):
+        oracle_sample(w, q_blocks=2)
+    times, desc = [], ""
+    for _ in range(max(1, args.steps)):
+        t, desc, _ = oracle_sample(w, q_blocks=32)
+        times.append(t)
+    t_layer = float(np.median(times))
+    value = dense_flops(w) / t_layer / 1e12
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": t_layer * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "keep_pct": w.keep_pct, "protect_pct": w.protect_pct},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------------------ our arm
+def run_ours(args, w):
+    from paper_2608_15522_b200 import binding as av
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the path has no CPU fallback")
+    av.load_library()
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=dev)
+
+    seed = rank      # every rank owns an independent layer (replica): weak scaling, no collective on the data path
+    q, k, v = wl.make_self_qkv(w, seed, dev)
+    qa, kc, vc = wl.make_cross_qkv(w, seed, dev)
+    n_protect = av.avsa_count_from_percent(w.protect_pct, w.n_video)
+    k_keep = max(1, av.avsa_count_from_percent(w.keep_pct, w.n_blocks))
+    gamma = 1.0 / (w.H * w.n_audio)
+    NB = w.n_blocks
+
+    # every buffer is allocated once, outside the timed region
+    o_a, lse, s, ws1 = av.avsa_cross_attn_scores(qa, kc, vc, score_gamma=gamma)
+    m = av.avsa_build_block_mask(q, k, s, n_protect, k_keep, w.blk)
+    o, _, ws3 = av.avsa_sparse_self_attn(q, k, v, m["col_idx"], m["col_cnt"], w.blk)
+    for ws in (ws1, m["ws"], ws3):
+        code, detail = av.avsa_read_status(ws)
+        if code != av.AVSA_OK:
+            raise RuntimeError(f"device status {av.status_string(code)} {detail}")
+    pairs = int(m["col_cnt"].sum().item())
+    prot_blocks = int(m["prot_blk"].sum().item())
+
+    def step():
+        av.avsa_cross_attn_scores(qa, kc, vc, scores=s, score_gamma=gamma, o=o_a, lse=lse, ws=ws1)
+        av.avsa_build_block_mask(q, k, s, n_protect, k_keep, w.blk, out=m, ws=m["ws"])
+        av.avsa_sparse_self_attn(q, k, v, m["col_idx"], m["col_cnt"], w.blk, o=o, ws=ws3)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    if sampler:
+        sampler.start()
+        time.sleep(0.3)
+    # ---- timed region: K whole steps; per-kernel events ride in the same stream
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    start.record()
+    for i in range(args.steps):
+        ev[i][0].record()
+        av.avsa_cross_attn_scores(qa, kc, vc, scores=s, score_gamma=gamma, o=o_a, lse=lse, ws=ws1)
+        ev[i][1].record()
+        av.avsa_build_block_mask(q, k, s, n_protect, k_keep, w.blk, out=m, ws=m["ws"])
+        ev[i][2].record()
+        av.avsa_sparse_self_attn(q, k, v, m["col_idx"], m["col_cnt"], w.blk, o=o, ws=ws3)
+        ev[i][3].record()
+    end.record()
+    barrier()
+    total_ms = start.elapsed_time(end)
+    t_cross = float(np.mean([e[0].elapsed_time(e[1]) for e in ev]))
+    t_mask = float(np.mean([e[1].elapsed_time(e[2]) for e in ev]))
+    t_attn = float(np.mean([e[2].elapsed_time(e[3]) for e in ev]))
+    clocks = sampler.stop() if sampler else None
+
+    # ---- dense baselines on the same tensors (outside the timed region)
+    idx_all = torch.arange(NB, dtype=torch.int32, device=dev).expand(w.B, w.H, NB, NB).contiguous()
+    cnt_all = torch.full((w.B, w.H, NB), NB, dtype=torch.int32, device=dev)
+
+    def time_fn(fn, n):
+        fn(); torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(n):
+            fn()
+        b.record(); torch.cuda.synchronize()
+        return a.elapsed_time(b) / n
+
+    t_dense_ours = time_fn(lambda: av.avsa_sparse_self_attn(q, k, v, idx_all, cnt_all, w.blk, o=o, ws=ws3), 3)
+    try:
+        t_dense_lib = time_fn(lambda: torch.nn.functional.scaled_dot_product_attention(q, k, v), 3)
+    except Exception:
+        t_dense_lib = None
+    del idx_all, cnt_all
+
+    # ---- end to end through the public API with host buffers (pinned), copies inside the timed region
+    host_in = [t.cpu().pin_memory() for t in (qa, kc, vc, q, k, v)]
+    host_out = torch.empty(o.shape, dtype=o.dtype).pin_memory()
+    dev_in = [qa, kc, vc, q, k, v]
+    h2d = sum(t.numel() * t.element_size() for t in host_in)
+    d2h = host_out.numel() * host_out.element_size()
+
+    def e2e_step():
+        for d_t, h_t in zip(dev_in, host_in):
+            d_t.copy_(h_t, non_blocking=True)
+        step()
+        host_out.copy_(o, non_blocking=True)
+
+    e2e_step(); barrier()
+    e2e_steps = max(2, min(args.steps, 5))
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(e2e_steps):
+        e2e_step()
+    b.record()
+    barrier()
+    e2e_ms = a.elapsed_time(b) / e2e_steps
+
+    # ---- max over ranks
+    times = torch.tensor([total_ms, e2e_ms], dtype=torch.float64, device=dev)
+    if dist is not None:
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+    total_ms, e2e_ms = float(times[0]), float(times[1])
+    ms_per_step = total_ms / args.steps
+    if rank == 0:
+        peaks, peak_kind = load_peaks()
+        fl_dense = dense_flops(w)
+        fl_exec = pairs * 4.0 * w.blk * w.blk * w.d
+        value = world * fl_dense / (ms_per_step * 1e-3) / 1e12
+        achieved = fl_exec / (t_attn * 1e-3) / 1e12
+        peak = float(peaks.get("bf16_tflops", FALLBACK_PEAKS["bf16_tflops"]))
+        sustained = float(peaks.get("bf16_tflops_sustained", FALLBACK_PEAKS["bf16_tflops_sustained"]))
+        hbm = float(peaks.get("hbm_gbs", FALLBACK_PEAKS["hbm_gbs"]))
+        mask_bytes = 2.0 * w.B * w.H * w.n_video * w.d * 2 + 3.0 * w.B * w.H * NB * NB * 4
+        cross_bytes = 2.0 * w.B * w.H * w.n_video * w.d * 2
+        dense_best = min(x for x in (t_dense_ours, t_dense_lib) if x is not None)
+        cores = len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else os.cpu_count()
+        if args.no_cpu_baseline:
+            cpu = None
+        else:
+            t_cpu, desc, _ = oracle_sample(w, q_blocks=w.n_blocks)
+            cpu = {"value": fl_dense / t_cpu / 1e12, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc}
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": w.name, "B": w.B, "H": w.H, "d": w.d, "n_video": w.n_video, "n_audio": w.n_audio,
+                       "blk": w.blk, "keep_pct": w.keep_pct, "protect_pct": w.protect_pct, "k_keep": k_keep,
+                       "n_protect": n_protect, "protected_blocks": prot_blocks, "n_blocks": NB,
+                       "executed_pair_fraction": pairs / float(w.B * w.H * NB * NB),
+                       "l2": "inputs (Q,K,V of both attentions, 1.2 GB) are larger than the 126 MB L2; no flush",
+                       "multi_gpu": "independent replica per GPU, no data-path collective"},
+            "ms": {"cross_attn_scores": t_cross, "build_block_mask": t_mask, "sparse_self_attn": t_attn,
+                   "dense_keep_all_ours": t_dense_ours, "dense_library_sdpa": t_dense_lib},
+            "speedup_vs_dense": {"attn_only": dense_best / t_attn, "layer_step": dense_best / ms_per_step,
+                                 "dense_is": "library_sdpa" if dense_best == t_dense_lib else "keep_all_ours"},
+            "executed_tflops": achieved,
+            "roofline": {"kernel": "attn_fwd_kernel<128,128,MODE_LIST> (avsa_sparse_self_attn)", "bound": "tensor",
+                         "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
+                         "peak_source": f"{peak_kind} bf16_tflops (burst)", "frac_of_sustained": achieved / sustained,
+                         "frac_of_nominal_2250": achieved / 2250.0,
+                         "traffic": NCU_TRAFFIC_BYTES.get(w.name)},
+            "hbm_kernels": {"build_block_mask_gbs": mask_bytes / (t_mask * 1e-3) / 1e9,
+                            "build_block_mask_frac": mask_bytes / (t_mask * 1e-3) / 1e9 / hbm,
+                            "cross_attn_scores_gbs": cross_bytes / (t_cross * 1e-3) / 1e9,
+                            "cross_attn_scores_frac": cross_bytes / (t_cross * 1e-3) / 1e9 / hbm,
+                            "peak_gbs": hbm, "peak_source": peak_kind},
+            "cpu_baseline": cpu,
+            "e2e": {"value": world * fl_dense / (e2e_ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
+                    "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+            "gpu_launches": KERNELS_PER_STEP * args.steps,
+            "clocks": clocks,
+        }
+        print(json.dumps(line))
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="ovi", choices=wl.all_workload_names())
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    w = wl.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_ours(args, w)
+
+
+if __name__ == "__main__":
+    main()
