@@ -163,8 +163,11 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__
 
   const int n_tiles[2] = {(cnt + 1) >> 1, cnt >> 1};
 
+  // The four service warps (0-3) give registers to the eight softmax warps (4-11); each role
+  // changes its own budget as the first thing it does.
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 64;");
     if (lane == 0) {
       mbar_expect_tx(BAR(Q_FULL), BLK * D * 2);
       for (int pn = 0; pn < NPANEL; pn++)
@@ -199,6 +202,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 64;");
     if (lane == 0) {
       const uint32_t idesc_qk = make_idesc_bf16(128, BLK, 0, 0);
       const uint32_t idesc_pv = make_idesc_bf16(128, D, 0, 1);
@@ -238,8 +242,11 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__
       }
       if (ok) umma_commit(BAR(FINAL));
     }
-  } else if (warp >= 4) {
+  } else if (warp < 4) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 64;");
+  } else {
     // ------------------------------------------------------------------ softmax groups + epilogue
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 216;");
     const int w = (warp - 4) >> 2;               // group
     const int row = ((warp & 3) << 5) + lane;    // row of the tile == TMEM lane
     const uint32_t lane_off = static_cast<uint32_t>((warp & 3) * 32) << 16;
@@ -263,9 +270,14 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__
         for (int j = 0; j < BLK; j++)
           if (j >= ragged_valid) s[j] = 0xff800000u;
       }
-      float mx = -INFINITY;
+      float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // four independent chains
 #pragma unroll
-      for (int j = 0; j < BLK; j++) mx = fmaxf(mx, __uint_as_float(s[j]));
+      for (int j = 0; j < BLK; j += 8) {
+#pragma unroll
+        for (int u = 0; u < 4; u++)
+          mx4[u] = max3f(mx4[u], __uint_as_float(s[j + 2 * u]), __uint_as_float(s[j + 2 * u + 1]));
+      }
+      const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
       const float m_new = fmaxf(m_run, mx * p.scale_log2);
       const bool need = (m_new - m_run) > kRescaleThreshold;     // true on the first tile (m_run = -inf)
       float factor = 1.f;
@@ -286,20 +298,27 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__
         }
       }
       l_run *= factor;
-      float sum = 0.f;
-      const float neg_m = -m_run;
+      // p = exp2(s * c - m) on pairs: one packed FMA, two EX2, one packed add, one bf16x2 convert per pair
+      const uint64_t c2 = pack_f32x2(p.scale_log2, p.scale_log2);
+      const uint64_t nm2 = pack_f32x2(-m_run, -m_run);
+      uint64_t sum2[4] = {0ull, 0ull, 0ull, 0ull};
 #pragma unroll
       for (int c = 0; c < BLK / 32; c++) {
         uint32_t pk[16];
 #pragma unroll
         for (int j = 0; j < 16; j++) {
-          const float p0 = fast_exp2(fmaf(__uint_as_float(s[c * 32 + 2 * j]), p.scale_log2, neg_m));
-          const float p1 = fast_exp2(fmaf(__uint_as_float(s[c * 32 + 2 * j + 1]), p.scale_log2, neg_m));
-          sum += p0 + p1;
+          float x0, x1;
+          unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(s[c * 32 + 2 * j]), __uint_as_float(s[c * 32 + 2 * j + 1])),
+                                 c2, nm2), x0, x1);
+          const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
+          sum2[j & 3] = add_f32x2(sum2[j & 3], pack_f32x2(p0, p1));
           pk[j] = pack_bf16x2(p0, p1);
         }
         tmem_st16(TM_S[w] + lane_off + c * 16, pk);
       }
+      float sa, sb;
+      unpack_f32x2(add_f32x2(add_f32x2(sum2[0], sum2[1]), add_f32x2(sum2[2], sum2[3])), sa, sb);
+      const float sum = sa + sb;
       l_run += sum;
       tmem_wait_st();
       tc_fence_before();
