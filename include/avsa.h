@@ -123,6 +123,33 @@ AVSA_API int avsa_sparse_self_attn(int B, int H, int N, int d, int blk, avsa_bf1
                           float softmax_scale, void* ws, size_t ws_bytes, void* stream);
 AVSA_API size_t avsa_sparse_self_attn_workspace_bytes(int B, int H, int N, int d, int blk);
 
+/*
+ * Allocation-free variant of avsa_build_block_mask.  The paper has no counterpart; this is a
+ * convenience of the library for callers that have no device allocator to draw a workspace from:
+ * code that runs after its host application has frozen its memory budget, extensions loaded into
+ * a runtime that owns all device memory and hands none out, and latency-critical loops in which a
+ * synchronising allocation is not acceptable.
+ *
+ * Same arguments and results as avsa_build_block_mask, without `ws`: the scratch (pooled block means,
+ * fallback flag buffers and the status record) lives in a fixed array of AVSA_STATIC_SCRATCH_BYTES
+ * inside the library, which every GPU that loads libavsa.so holds until the process exits.
+ *   - Shapes whose avsa_build_block_mask_workspace_bytes() exceeds AVSA_STATIC_SCRATCH_BYTES are
+ *     refused with AVSA_ERR_WORKSPACE and nothing is enqueued.
+ *   - The first call on each device looks up the array's device address (with that device current).
+ *     Make that first call before starting any stream capture.
+ *   - The call allocates nothing: no cudaMalloc/cudaFree, no allocating library routine.
+ *   - All calls on a device share the one array, and it keeps the previous call's contents; what must
+ *     start from zero (the status record) is cleared by the call itself.  Two such calls that overlap
+ *     on the GPU (different streams) race on the array: serialise them.
+ *   - The mask kernels have no device-side failure mode (no waits, no list input), so there is no
+ *     status record to read after this call.
+ */
+#define AVSA_STATIC_SCRATCH_BYTES (16u << 20)
+AVSA_API int avsa_build_block_mask_static(int B, int H, int N, int d, int blk, avsa_bf16_4d q, avsa_bf16_4d k,
+                                          const float* scores, int n_protect, int k_keep, unsigned flags,
+                                          float softmax_scale, float* block_scores, int32_t* col_idx,
+                                          int32_t* col_cnt, uint8_t* prot_tok, uint8_t* prot_blk, void* stream);
+
 /* Host integer ceil(pct/100 * n): the count forms of rho and kappa (Eq. 8's ceiling). */
 AVSA_API int avsa_count_from_percent(int pct, int n);
 

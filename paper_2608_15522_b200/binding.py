@@ -29,7 +29,7 @@ AVSA_USE_GIVEN_BLOCK_SCORES = 4
 
 EXPORTS = (
     "avsa_cross_attn_scores", "avsa_cross_attn_scores_workspace_bytes",
-    "avsa_build_block_mask", "avsa_build_block_mask_workspace_bytes",
+    "avsa_build_block_mask", "avsa_build_block_mask_workspace_bytes", "avsa_build_block_mask_static",
     "avsa_sparse_self_attn", "avsa_sparse_self_attn_workspace_bytes",
     "avsa_count_from_percent", "avsa_read_status", "avsa_status_string", "avsa_version",
 )
@@ -68,6 +68,8 @@ def load_library() -> ctypes.CDLL:
     lib.avsa_build_block_mask.restype = i
     lib.avsa_build_block_mask_workspace_bytes.argtypes = [i, i, i, i, i]
     lib.avsa_build_block_mask_workspace_bytes.restype = sz
+    lib.avsa_build_block_mask_static.argtypes = [i, i, i, i, i, T, T, vp, i, i, u, f, vp, vp, vp, vp, vp, vp]
+    lib.avsa_build_block_mask_static.restype = i
     lib.avsa_sparse_self_attn.argtypes = [i, i, i, i, i, T, T, T, vp, vp, vp, vp, f, vp, sz, vp]
     lib.avsa_sparse_self_attn.restype = i
     lib.avsa_sparse_self_attn_workspace_bytes.argtypes = [i, i, i, i, i]
@@ -209,6 +211,28 @@ def avsa_build_block_mask(q, k, scores, n_protect, k_keep, blk, flags=AVSA_PROTE
                                    _ptr(prot_tok), _ptr(prot_blk), _ptr(ws), ws.numel(), _stream(dev))
     _check(st, "avsa_build_block_mask")
     return dict(block_scores=block_scores, col_idx=col_idx, col_cnt=col_cnt, prot_tok=prot_tok, prot_blk=prot_blk, ws=ws)
+
+
+AVSA_STATIC_SCRATCH_BYTES = 16 << 20
+
+
+def avsa_build_block_mask_static(q, k, scores, n_protect, k_keep, blk, out, flags=AVSA_PROTECT_ROWS, softmax_scale=0.0):
+    """avsa_build_block_mask without a workspace: the library's built-in scratch array is used.
+
+    For callers that must not allocate.  Accordingly this wrapper allocates nothing either: every output
+    tensor (block_scores, col_idx, col_cnt, prot_tok, prot_blk) must be supplied in ``out``.  Shapes that
+    need more scratch than AVSA_STATIC_SCRATCH_BYTES raise AvsaError(AVSA_ERR_WORKSPACE).  The first call
+    on a device resolves the array's address; make it before any stream capture.  Calls share the array, so
+    do not let two of them overlap on the GPU.
+    """
+    lib = load_library()
+    B, H, N, d = q.shape
+    st = lib.avsa_build_block_mask_static(B, H, N, d, blk, _t4(q), _t4(k), _ptr(scores), int(n_protect), int(k_keep),
+                                          int(flags), float(softmax_scale), _ptr(out["block_scores"]),
+                                          _ptr(out["col_idx"]), _ptr(out["col_cnt"]), _ptr(out["prot_tok"]),
+                                          _ptr(out["prot_blk"]), _stream(q.device))
+    _check(st, "avsa_build_block_mask_static")
+    return out
 
 
 def avsa_sparse_self_attn_workspace_bytes(B, H, N, d, blk) -> int:

@@ -1,6 +1,8 @@
 // Mask construction: protected token set (Eq. 3 / Eq. 8), block mean-pooling and block scores of the
 // base sparse pattern, per-(head, query block) top-k, and the protected block mask of Eq. 9 emitted
 // as ascending column lists.  CUDA-core kernels: the work is HBM- or latency-bound.
+#include <mutex>
+
 #include "avsa_common.cuh"
 
 namespace avsa {
@@ -390,4 +392,45 @@ extern "C" int avsa_build_block_mask(int B, int H, int N, int d, int blk, avsa_b
                                                              (flags & AVSA_PROTECT_COLS) ? 1 : 0, total_rows, col_idx,
                                                              col_cnt);
   return cudaGetLastError() == cudaSuccess ? AVSA_OK : AVSA_ERR_CUDA;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Allocation-free variant: the workspace is a fixed array in the library's own device image.
+// ------------------------------------------------------------------------------------------------
+static __device__ __align__(256) unsigned char g_static_mask_scratch[AVSA_STATIC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+void* g_static_scratch_addr[kMaxDevices] = {};   // device address of the array, per device ordinal
+std::mutex g_static_scratch_mutex;
+
+// In host code the array's name is only a handle for the runtime; the address a kernel can use comes
+// from cudaGetSymbolAddress, asked once per device with that device current.
+int static_scratch_for_current_device(void** out) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return AVSA_ERR_CUDA;
+  if (dev < 0 || dev >= kMaxDevices) return AVSA_ERR_UNSUPPORTED;
+  std::lock_guard<std::mutex> lock(g_static_scratch_mutex);
+  if (g_static_scratch_addr[dev] == nullptr) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_static_mask_scratch) != cudaSuccess || ptr == nullptr) return AVSA_ERR_CUDA;
+    g_static_scratch_addr[dev] = ptr;
+  }
+  *out = g_static_scratch_addr[dev];
+  return AVSA_OK;
+}
+}  // namespace
+
+extern "C" int avsa_build_block_mask_static(int B, int H, int N, int d, int blk, avsa_bf16_4d q, avsa_bf16_4d k,
+                                            const float* scores, int n_protect, int k_keep, unsigned flags,
+                                            float softmax_scale, float* block_scores, int32_t* col_idx,
+                                            int32_t* col_cnt, uint8_t* prot_tok, uint8_t* prot_blk, void* stream) {
+  if (B <= 0 || H <= 0 || N <= 0 || d <= 0 || blk <= 0) return AVSA_ERR_INVALID_ARG;
+  const size_t need = avsa_build_block_mask_workspace_bytes(B, H, N, d, blk);
+  if (need == 0 || need > static_cast<size_t>(AVSA_STATIC_SCRATCH_BYTES)) return AVSA_ERR_WORKSPACE;
+  void* scratch = nullptr;
+  const int rc = static_scratch_for_current_device(&scratch);
+  if (rc != AVSA_OK) return rc;
+  return avsa_build_block_mask(B, H, N, d, blk, q, k, scores, n_protect, k_keep, flags, softmax_scale, block_scores,
+                               col_idx, col_cnt, prot_tok, prot_blk, scratch, AVSA_STATIC_SCRATCH_BYTES, stream);
 }
