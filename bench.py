@@ -35,7 +35,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the sparse attention kernel, from the ncu capture
 # summarised under profiles/ (None until a capture exists for that workload)
 NCU_TRAFFIC_BYTES = {}
-KERNELS_PER_STEP = 12   # cross: clear, pass 1, merge, pass 2, head sum; mask: clear, select, pool, scores, rows; attn: clear, attn
+KERNELS_PER_STEP = 11   # cross: clear, pass 1, merge, pass 2, head sum; mask: select, pool, scores, rows; attn: clear, attn
 
 
 def load_peaks():

@@ -30,6 +30,7 @@ __global__ void __launch_bounds__(256) pool_kernel(const __nv_bfloat16* __restri
   constexpr int TPR = D / 8;          // threads per row
   constexpr int RPP = 256 / TPR;      // rows per pass
   __shared__ float part[RPP][D + 4];
+
   const int nb = blockIdx.x, bh = blockIdx.y, which = blockIdx.z;
   const int b = bh / H, h = bh % H;
   const __nv_bfloat16* src = which == 0 ? q + b * q_sb + h * q_sh : k + b * k_sb + h * k_sh;
@@ -72,56 +73,93 @@ __global__ void __launch_bounds__(256) pool_kernel(const __nv_bfloat16* __restri
 }
 
 // ------------------------------------------------------------------------------------------------
-// (ii) block scores Bs[bh, i, j] = qbar[bh,i,:] . kbar[bh,j,:] * scale.  64x64 tile per CTA,
-// 256 threads x (4x4) outputs, channels summed in ascending order.
+// (ii) block scores Bs[bh, i, j] = qbar[bh,i,:] . kbar[bh,j,:] * scale.  64x64 tile per CTA; both
+// operand tiles are brought into shared memory in one shot (all loads in flight at once), stored
+// channel-major so that each thread reads its 4 rows / 4 columns as one float4; 128 threads x (8x4)
+// outputs, channels summed in ascending order.
 // ------------------------------------------------------------------------------------------------
+constexpr int kScorePitch = 64 + 4;
 template <int D>
-__global__ void __launch_bounds__(256) block_score_kernel(const float* __restrict__ qbar,
+__global__ void __launch_bounds__(128) block_score_kernel(const float* __restrict__ qbar,
                                                           const float* __restrict__ kbar, float* __restrict__ bs,
                                                           int NB, float scale) {
-  constexpr int KC = 32;
-  __shared__ float sq[KC][64 + 1];
-  __shared__ float sk[KC][64 + 1];
+  extern __shared__ __align__(16) float score_smem[];
+  float(*sq)[kScorePitch] = reinterpret_cast<float(*)[kScorePitch]>(score_smem);
+  float(*sk)[kScorePitch] = reinterpret_cast<float(*)[kScorePitch]>(score_smem + D * kScorePitch);
   const int bh = blockIdx.z, i0 = blockIdx.y * 64, j0 = blockIdx.x * 64;
   const float* qb = qbar + static_cast<int64_t>(bh) * NB * D;
   const float* kb = kbar + static_cast<int64_t>(bh) * NB * D;
-  const int tx = threadIdx.x % 16, ty = threadIdx.x / 16;
-  float acc[4][4];
+  // Launched as an ordinary stream-ordered kernel: it starts only after both the token select and the
+  // pooling kernel (which may overlap each other) have finished.  The list kernel behind it may be
+  // scheduled early and waits for this grid.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+#pragma unroll 1
+  for (int half = 0; half < 2; half++) {
+    const int r = threadIdx.x % 64, cg = threadIdx.x / 64 + 2 * half;
+    float4 vq[D / 16], vk[D / 16];
 #pragma unroll
-  for (int a = 0; a < 4; a++)
+    for (int it = 0; it < D / 16; it++) {
+      const int c4 = cg + 4 * it;
+      vq[it] = (i0 + r < NB) ? __ldg(reinterpret_cast<const float4*>(qb + static_cast<int64_t>(i0 + r) * D) + c4)
+                             : make_float4(0.f, 0.f, 0.f, 0.f);
+      vk[it] = (j0 + r < NB) ? __ldg(reinterpret_cast<const float4*>(kb + static_cast<int64_t>(j0 + r) * D) + c4)
+                             : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+#pragma unroll
+    for (int it = 0; it < D / 16; it++) {
+      const int c = (cg + 4 * it) * 4;
+      sq[c][r] = vq[it].x; sq[c + 1][r] = vq[it].y; sq[c + 2][r] = vq[it].z; sq[c + 3][r] = vq[it].w;
+      sk[c][r] = vk[it].x; sk[c + 1][r] = vk[it].y; sk[c + 2][r] = vk[it].z; sk[c + 3][r] = vk[it].w;
+    }
+  }
+  __syncthreads();
+  const int tx = threadIdx.x % 16, ty = threadIdx.x / 16;     // 16 x 8 threads, 8 rows x 4 columns each
+  float acc[8][4];
+#pragma unroll
+  for (int a = 0; a < 8; a++)
 #pragma unroll
     for (int c = 0; c < 4; c++) acc[a][c] = 0.f;
-  for (int k0 = 0; k0 < D; k0 += KC) {
-    for (int e = threadIdx.x; e < 64 * KC; e += 256) {
-      const int r = e / KC, c = e % KC;
-      sq[c][r] = (i0 + r < NB) ? qb[static_cast<int64_t>(i0 + r) * D + k0 + c] : 0.f;
-      sk[c][r] = (j0 + r < NB) ? kb[static_cast<int64_t>(j0 + r) * D + k0 + c] : 0.f;
-    }
-    __syncthreads();
+#pragma unroll 4
+  for (int c = 0; c < D; c++) {
+    const float4 a0 = *reinterpret_cast<const float4*>(&sq[c][ty * 8]);
+    const float4 a1 = *reinterpret_cast<const float4*>(&sq[c][ty * 8 + 4]);
+    const float4 bv = *reinterpret_cast<const float4*>(&sk[c][tx * 4]);
+    const float a[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+    const float bq[4] = {bv.x, bv.y, bv.z, bv.w};
 #pragma unroll
-    for (int c = 0; c < KC; c++) {
-      float a[4], bq[4];
+    for (int t = 0; t < 8; t++)
 #pragma unroll
-      for (int t = 0; t < 4; t++) {
-        a[t] = sq[c][ty * 4 + t];
-        bq[t] = sk[c][tx * 4 + t];
-      }
-#pragma unroll
-      for (int t = 0; t < 4; t++)
-#pragma unroll
-        for (int u = 0; u < 4; u++) acc[t][u] = fmaf(a[t], bq[u], acc[t][u]);
-    }
-    __syncthreads();
+      for (int u = 0; u < 4; u++) acc[t][u] = fmaf(a[t], bq[u], acc[t][u]);
   }
 #pragma unroll
-  for (int t = 0; t < 4; t++) {
-    const int i = i0 + ty * 4 + t;
+  for (int t = 0; t < 8; t++) {
+    const int i = i0 + ty * 8 + t;
     if (i >= NB) continue;
+    float* dst = bs + (static_cast<int64_t>(bh) * NB + i) * NB + j0 + tx * 4;
+    if (j0 + tx * 4 + 3 < NB && (NB & 3) == 0) {
+      *reinterpret_cast<float4*>(dst) = make_float4(acc[t][0] * scale, acc[t][1] * scale, acc[t][2] * scale,
+                                                    acc[t][3] * scale);
+    } else {
 #pragma unroll
-    for (int u = 0; u < 4; u++) {
-      const int j = j0 + tx * 4 + u;
-      if (j < NB) bs[(static_cast<int64_t>(bh) * NB + i) * NB + j] = acc[t][u] * scale;
+      for (int u = 0; u < 4; u++)
+        if (j0 + tx * 4 + u < NB) dst[u] = acc[t][u] * scale;
     }
+  }
+}
+
+// Adds one warp's digits to a shared-memory histogram.  When every participating lane holds the same
+// digit (the usual case for the leading byte of like-signed scores) one lane adds the whole count;
+// otherwise each lane adds its own (the hardware serialises only lanes that really collide).
+__device__ __forceinline__ void warp_hist_add(int* bins, bool in, uint32_t dgt, int lane) {
+  const unsigned inmask = __ballot_sync(0xffffffffu, in);
+  if (inmask == 0u) return;
+  const int leader = __ffs(inmask) - 1;
+  const uint32_t d0 = __shfl_sync(0xffffffffu, dgt, leader);
+  const bool uniform = __all_sync(0xffffffffu, !in || dgt == d0);
+  if (uniform) {
+    if (lane == leader) atomicAdd(&bins[d0], __popc(inmask));
+  } else if (in) {
+    atomicAdd(&bins[dgt], 1);
   }
 }
 
@@ -129,7 +167,8 @@ __global__ void __launch_bounds__(256) block_score_kernel(const float* __restric
 // Radix-select helper: given 256 digit counts (descending scan), find the digit that holds the
 // want-th largest element.  One warp; lane l owns digits 255-8l .. 248-8l.
 // ------------------------------------------------------------------------------------------------
-__device__ __forceinline__ void warp_pick_digit(const int* bins, int want, int lane, int& digit, int& above) {
+__device__ __forceinline__ void warp_pick_digit(const int* bins, int want, int lane, int& digit, int& above,
+                                                int& in_bin) {
   int local[8];
   int sum = 0;
 #pragma unroll
@@ -145,7 +184,7 @@ __device__ __forceinline__ void warp_pick_digit(const int* bins, int want, int l
   }
   const int excl = incl - sum;
   const bool mine = (excl < want) && (want <= incl);
-  int dg = 0, ab = 0;
+  int dg = 0, ab = 0, ib = 0;
   if (mine) {
     int run = excl;
 #pragma unroll
@@ -153,6 +192,7 @@ __device__ __forceinline__ void warp_pick_digit(const int* bins, int want, int l
       if (run < want && want <= run + local[i]) {
         dg = 255 - (lane * 8 + i);
         ab = run;
+        ib = local[i];
       }
       run += local[i];
     }
@@ -161,100 +201,124 @@ __device__ __forceinline__ void warp_pick_digit(const int* bins, int want, int l
   const int src = __ffs(who) - 1;
   digit = __shfl_sync(0xffffffffu, dg, src);
   above = __shfl_sync(0xffffffffu, ab, src);
+  in_bin = __shfl_sync(0xffffffffu, ib, src);
 }
 
 // ------------------------------------------------------------------------------------------------
-// (iii) protected token set: one CTA of 1024 threads per batch item.  Radix select (4 x 8 bits) of
-// the n_protect-th largest key, then an index-ordered pass that takes every larger key and the
-// lowest-index ties, writes the token flags and raises the flag of every block that holds one.
+// (iii) protected token set: one CTA of 1024 threads per batch item.  The canonical keys are staged
+// in shared memory once (global memory is re-read instead when they do not fit); a radix select
+// (4 x 8 bits, warp-aggregated histogram) finds the n_protect-th largest key; then every warp walks
+// its own contiguous segment in index order, taking every larger key and the lowest-index ties,
+// writes the token flags and raises the flag of every block that holds one.  Block 0 also resets
+// the status record of the call.
 // ------------------------------------------------------------------------------------------------
+constexpr int kSelectSmemKeys = 56 * 1024;   // 224 KB of keys at most
+
+template <bool STAGED>
 __global__ void __launch_bounds__(1024) token_select_kernel(const float* __restrict__ scores, int N, int n_protect,
                                                             int blk, int NB, uint8_t* __restrict__ prot_tok,
-                                                            uint8_t* __restrict__ prot_blk) {
+                                                            uint8_t* __restrict__ prot_blk, StatusRecord* status) {
+  extern __shared__ uint32_t skeys[];
   __shared__ int bins[256];
-  __shared__ int s_digit, s_above;
+  __shared__ int s_digit, s_above, s_in_bin;
   __shared__ int warp_cnt[32];
-  __shared__ int s_eq_seen;
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const float* s = scores + static_cast<int64_t>(b) * N;
   uint8_t* ptok = prot_tok + static_cast<int64_t>(b) * N;
   uint8_t* pblk = prot_blk + static_cast<int64_t>(b) * NB;
+  // nothing launched next on the stream depends on this kernel until the list emission, so let the
+  // pooling kernel start right away (programmatic dependent launch)
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  if (b == 0 && tid == 0) {
+    status->code = 0;
+    status->where = 0;
+    status->item = 0;
+    status->aux = 0;
+  }
   for (int i = tid; i < NB; i += 1024) pblk[i] = 0;
   if (n_protect <= 0) {
     for (int i = tid; i < N; i += 1024) ptok[i] = 0;
     return;
   }
+  if (STAGED) {
+#pragma unroll 8
+    for (int i = tid; i < N; i += 1024) skeys[i] = rank_key(__ldg(s + i));
+  }
+  auto key_at = [&](int i) -> uint32_t { return STAGED ? skeys[i] : rank_key(__ldg(s + i)); };
   uint32_t prefix = 0, mask = 0;
   int want = n_protect;
   for (int pass = 0; pass < 4; pass++) {
     const int shift = 24 - 8 * pass;
     if (tid < 256) bins[tid] = 0;
-    __syncthreads();
+    __syncthreads();     // also orders the staging stores before the first reads
     for (int i0 = 0; i0 < N; i0 += 1024) {
       const int i = i0 + tid;
       const bool valid = i < N;
-      const uint32_t key = valid ? rank_key(s[i]) : 0u;
+      const uint32_t key = valid ? key_at(i) : 0u;
       const bool in = valid && ((key & mask) == prefix);
-      const uint32_t dgt = in ? ((key >> shift) & 255u) : 256u;
-      const unsigned peers = __match_any_sync(0xffffffffu, dgt);
-      if (in && lane == __ffs(peers) - 1) atomicAdd(&bins[dgt], __popc(peers));
+      warp_hist_add(bins, in, (key >> shift) & 255u, lane);
     }
     __syncthreads();
     if (warp == 0) {
-      int dg, ab;
-      warp_pick_digit(bins, want, lane, dg, ab);
+      int dg, ab, ib;
+      warp_pick_digit(bins, want, lane, dg, ab, ib);
       if (lane == 0) {
         s_digit = dg;
         s_above = ab;
+        s_in_bin = ib;
       }
     }
     __syncthreads();
     want -= s_above;
     prefix |= static_cast<uint32_t>(s_digit) << shift;
     mask |= 255u << shift;
+    const bool whole_bin = (s_in_bin == want);   // every key of the bin is taken: no need to refine further
     __syncthreads();
+    if (whole_bin) break;
   }
   const uint32_t T = prefix;     // the n_protect-th largest key; `want` ties at T are taken, lowest index first
-  if (tid == 0) s_eq_seen = 0;
+  // contiguous, 32-aligned segment per warp
+  const int seg = ((N + 31) / 32 + 31) / 32 * 32;
+  const int lo = warp * seg, hi = min(N, lo + seg);
+  int eq_mine = 0;
+  for (int i0 = lo; i0 < hi; i0 += 32) {
+    const int i = i0 + lane;
+    eq_mine += __popc(__ballot_sync(0xffffffffu, i < hi && key_at(i) == T));
+  }
+  if (lane == 0) warp_cnt[warp] = eq_mine;
   __syncthreads();
-  for (int i0 = 0; i0 < N; i0 += 1024) {
-    const int i = i0 + tid;
-    const bool valid = i < N;
-    const uint32_t key = valid ? rank_key(s[i]) : 0u;
+  int eq_seen = 0;
+  for (int w2 = 0; w2 < warp; w2++) eq_seen += warp_cnt[w2];
+  for (int i0 = lo; i0 < hi; i0 += 32) {
+    const int i = i0 + lane;
+    const bool valid = i < hi;
+    const uint32_t key = valid ? key_at(i) : 0u;
     const bool gt = valid && key > T;
     const bool eq = valid && key == T;
     const unsigned eqm = __ballot_sync(0xffffffffu, eq);
-    if (lane == 0) warp_cnt[warp] = __popc(eqm);
-    __syncthreads();
-    int before = s_eq_seen;
-    for (int w = 0; w < warp; w++) before += warp_cnt[w];
-    const int rank = before + __popc(eqm & ((1u << lane) - 1u));
-    const bool keep = gt || (eq && rank < want);
+    const bool keep = gt || (eq && (eq_seen + __popc(eqm & ((1u << lane) - 1u))) < want);
+    eq_seen += __popc(eqm);
     if (valid) ptok[i] = keep ? 1 : 0;
     const unsigned km = __ballot_sync(0xffffffffu, keep);
-    if (km != 0u && lane == 0) pblk[(i0 + warp * 32) / blk] = 1;   // blk is a multiple of 32
-    __syncthreads();
-    if (tid == 0) {
-      int tot = 0;
-      for (int w = 0; w < 32; w++) tot += warp_cnt[w];
-      s_eq_seen += tot;
-    }
-    __syncthreads();
+    if (km != 0u && lane == 0) pblk[i0 / blk] = 1;   // blk is a multiple of 32 and so is i0
   }
 }
 
 // ------------------------------------------------------------------------------------------------
 // (iv) per-(head, query block) top-k_keep of a block-score row, protection OR (Eq. 9), ascending
-// list emission.  One warp per row, 4 rows per CTA.
+// list emission.  One warp per row, 4 rows per CTA; the row's keys live in registers (KPL per lane,
+// element j*32+lane in slot j).  The radix select stops as soon as the bin that holds the k-th key
+// is taken whole.
 // ------------------------------------------------------------------------------------------------
+template <int KPL>
 __global__ void __launch_bounds__(128) row_select_kernel(const float* __restrict__ bs, const uint8_t* __restrict__ prot_blk,
                                                          int H, int NB, int k_keep, int protect_rows,
                                                          int protect_cols, int total_rows, int32_t* __restrict__ col_idx,
                                                          int32_t* __restrict__ col_cnt) {
-  extern __shared__ uint32_t dyn[];
+  __shared__ int all_bins[4][256];
+  asm volatile("griddepcontrol.wait;" ::: "memory");   // block scores and block flags come from earlier kernels
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  uint32_t* keys = dyn + static_cast<size_t>(warp) * NB;
-  int* bins = reinterpret_cast<int*>(dyn + static_cast<size_t>(4) * NB) + warp * 256;
+  int* bins = all_bins[warp];
   const int row = blockIdx.x * 4 + warp;      // row = (b*H + h)*NB + qb
   if (row >= total_rows) return;
   const int qb = row % NB;
@@ -264,49 +328,54 @@ __global__ void __launch_bounds__(128) row_select_kernel(const float* __restrict
   const uint8_t* pb = prot_blk + static_cast<int64_t>(b) * NB;
   const bool row_prot = protect_rows && pb[qb] != 0;
   const unsigned lt = (1u << lane) - 1u;
+  const bool keep_all = row_prot || k_keep >= NB;
 
+  uint32_t keys[KPL];
   uint32_t T = 0;
   int want = 0;
-  if (!row_prot && k_keep < NB) {
-    for (int i = lane; i < NB; i += 32) keys[i] = rank_key(src[i]);
-    __syncwarp();
+  if (!keep_all) {
+#pragma unroll
+    for (int j = 0; j < KPL; j++) {
+      const int i = j * 32 + lane;
+      keys[j] = (i < NB) ? rank_key(__ldg(src + i)) : 0u;
+    }
     uint32_t prefix = 0, mask = 0;
     want = k_keep;
     for (int pass = 0; pass < 4; pass++) {
       const int shift = 24 - 8 * pass;
-      for (int i = lane; i < 256; i += 32) bins[i] = 0;
+#pragma unroll
+      for (int i = 0; i < 8; i++) bins[i * 32 + lane] = 0;
       __syncwarp();
-      for (int i0 = 0; i0 < NB; i0 += 32) {
-        const int i = i0 + lane;
-        const bool valid = i < NB;
-        const uint32_t key = valid ? keys[i] : 0u;
-        const bool in = valid && ((key & mask) == prefix);
-        const uint32_t dgt = in ? ((key >> shift) & 255u) : 256u;
-        const unsigned peers = __match_any_sync(0xffffffffu, dgt);
-        if (in && lane == __ffs(peers) - 1) bins[dgt] += __popc(peers);
-        __syncwarp();
+#pragma unroll
+      for (int j = 0; j < KPL; j++) {
+        if (j * 32 < NB) {
+          const bool in = (j * 32 + lane < NB) && ((keys[j] & mask) == prefix);
+          warp_hist_add(bins, in, (keys[j] >> shift) & 255u, lane);
+        }
       }
-      int dg, ab;
-      warp_pick_digit(bins, want, lane, dg, ab);
+      __syncwarp();
+      int dg, ab, ib;
+      warp_pick_digit(bins, want, lane, dg, ab, ib);
       want -= ab;
       prefix |= static_cast<uint32_t>(dg) << shift;
       mask |= 255u << shift;
       __syncwarp();
+      if (ib == want) break;     // the whole bin is taken
     }
     T = prefix;
   }
-  const bool keep_all = row_prot || k_keep >= NB;
   int pos = 0, eq_seen = 0;
-  for (int i0 = 0; i0 < NB; i0 += 32) {
-    const int i = i0 + lane;
+#pragma unroll
+  for (int j = 0; j < KPL; j++) {
+    if (j * 32 >= NB) break;
+    const int i = j * 32 + lane;
     const bool valid = i < NB;
     bool keep;
     if (keep_all) {
       keep = valid;
     } else {
-      const uint32_t key = valid ? keys[i] : 0u;
-      const bool gt = valid && key > T;
-      const bool eq = valid && key == T;
+      const bool gt = valid && keys[j] > T;
+      const bool eq = valid && keys[j] == T;
       const unsigned eqm = __ballot_sync(0xffffffffu, eq);
       keep = gt || (eq && (eq_seen + __popc(eqm & lt)) < want);
       eq_seen += __popc(eqm);
@@ -368,29 +437,75 @@ extern "C" int avsa_build_block_mask(int B, int H, int N, int d, int blk, avsa_b
   uint8_t* pblk = prot_blk != nullptr ? prot_blk : base + w.pblk;
   const float scale = softmax_scale != 0.f ? softmax_scale : 1.0f / sqrtf(static_cast<float>(d));
 
-  clear_status_kernel<<<1, 1, 0, st>>>(static_cast<StatusRecord*>(ws));
-  token_select_kernel<<<B, 1024, 0, st>>>(scores, N, n_protect, blk, NB, ptok, pblk);
+  if (N <= kSelectSmemKeys) {
+    const size_t key_bytes = static_cast<size_t>(N) * sizeof(uint32_t);
+    if (cudaFuncSetAttribute(token_select_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             static_cast<int>(key_bytes)) != cudaSuccess)
+      return AVSA_ERR_CUDA;
+    token_select_kernel<true><<<B, 1024, key_bytes, st>>>(scores, N, n_protect, blk, NB, ptok, pblk,
+                                                         static_cast<StatusRecord*>(ws));
+  } else {
+    token_select_kernel<false><<<B, 1024, 0, st>>>(scores, N, n_protect, blk, NB, ptok, pblk,
+                                                   static_cast<StatusRecord*>(ws));
+  }
   if (!given) {
     const __nv_bfloat16* qp = static_cast<const __nv_bfloat16*>(q.ptr);
     const __nv_bfloat16* kp = static_cast<const __nv_bfloat16*>(k.ptr);
     dim3 pg(NB, B * H, 2);
     dim3 sg((NB + 63) / 64, (NB + 63) / 64, B * H);
+    // the pooling kernel does not read anything the token select writes: allow it to start early
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = pg;
+    cfg.blockDim = dim3(256, 1, 1);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = st;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    const int64_t qsb = q.stride_b, qsh = q.stride_h, qsn = q.stride_n, ksb = k.stride_b, ksh = k.stride_h,
+                  ksn = k.stride_n;
+    const size_t score_smem = static_cast<size_t>(2) * d * kScorePitch * sizeof(float);
+    cudaError_t e;
     if (d == 128) {
-      pool_kernel<128><<<pg, 256, 0, st>>>(qp, q.stride_b, q.stride_h, q.stride_n, kp, k.stride_b, k.stride_h,
-                                          k.stride_n, qbar, kbar, H, N, blk);
-      block_score_kernel<128><<<sg, 256, 0, st>>>(qbar, kbar, block_scores, NB, scale);
+      e = cudaLaunchKernelEx(&cfg, pool_kernel<128>, qp, qsb, qsh, qsn, kp, ksb, ksh, ksn, qbar, kbar, H, N, blk);
+      if (e != cudaSuccess) return AVSA_ERR_CUDA;
+      if (cudaFuncSetAttribute(block_score_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               static_cast<int>(score_smem)) != cudaSuccess)
+        return AVSA_ERR_CUDA;
+      block_score_kernel<128><<<sg, 128, score_smem, st>>>(qbar, kbar, block_scores, NB, scale);
     } else {
-      pool_kernel<64><<<pg, 256, 0, st>>>(qp, q.stride_b, q.stride_h, q.stride_n, kp, k.stride_b, k.stride_h,
-                                         k.stride_n, qbar, kbar, H, N, blk);
-      block_score_kernel<64><<<sg, 256, 0, st>>>(qbar, kbar, block_scores, NB, scale);
+      e = cudaLaunchKernelEx(&cfg, pool_kernel<64>, qp, qsb, qsh, qsn, kp, ksb, ksh, ksn, qbar, kbar, H, N, blk);
+      if (e != cudaSuccess) return AVSA_ERR_CUDA;
+      block_score_kernel<64><<<sg, 128, score_smem, st>>>(qbar, kbar, block_scores, NB, scale);
     }
   }
   const int total_rows = B * H * NB;
-  const size_t smem = (static_cast<size_t>(4) * NB + 4 * 256) * sizeof(uint32_t);
-  row_select_kernel<<<(total_rows + 3) / 4, 128, smem, st>>>(block_scores, pblk, H, NB, k_keep,
-                                                             (flags & AVSA_PROTECT_ROWS) ? 1 : 0,
-                                                             (flags & AVSA_PROTECT_COLS) ? 1 : 0, total_rows, col_idx,
-                                                             col_cnt);
+  const int pr = (flags & AVSA_PROTECT_ROWS) ? 1 : 0, pc = (flags & AVSA_PROTECT_COLS) ? 1 : 0;
+  const unsigned rgrid = static_cast<unsigned>((total_rows + 3) / 4);
+  {
+    cudaLaunchAttribute rattr[1];
+    rattr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    rattr[0].val.programmaticStreamSerializationAllowed = given ? 0 : 1;   // only behind the block-score kernel
+    cudaLaunchConfig_t rcfg = {};
+    rcfg.gridDim = dim3(rgrid, 1, 1);
+    rcfg.blockDim = dim3(128, 1, 1);
+    rcfg.dynamicSmemBytes = 0;
+    rcfg.stream = st;
+    rcfg.attrs = rattr;
+    rcfg.numAttrs = 1;
+    const float* bsc = block_scores;
+    const uint8_t* pbc = pblk;
+    cudaError_t e;
+    if (NB <= 256)
+      e = cudaLaunchKernelEx(&rcfg, row_select_kernel<8>, bsc, pbc, H, NB, k_keep, pr, pc, total_rows, col_idx, col_cnt);
+    else if (NB <= 512)
+      e = cudaLaunchKernelEx(&rcfg, row_select_kernel<16>, bsc, pbc, H, NB, k_keep, pr, pc, total_rows, col_idx, col_cnt);
+    else
+      e = cudaLaunchKernelEx(&rcfg, row_select_kernel<64>, bsc, pbc, H, NB, k_keep, pr, pc, total_rows, col_idx, col_cnt);
+    if (e != cudaSuccess) return AVSA_ERR_CUDA;
+  }
   return cudaGetLastError() == cudaSuccess ? AVSA_OK : AVSA_ERR_CUDA;
 }
 

@@ -102,6 +102,25 @@ def test_mask_ties_nan_and_signed_zero_bit_exact():
         assert np.array_equal(out["col_idx"].cpu().numpy(), idx), (n_protect, k_keep)
 
 
+def test_mask_long_sequence_beyond_the_shared_memory_key_cache():
+    """N above 57344 tokens: the token select re-reads global memory instead of staging keys on chip."""
+    B, H, N, d, blk = 2, 1, 60000 + 77, 128, 128
+    NB = (N + blk - 1) // blk
+    rng = np.random.default_rng(9)
+    bs = rng.standard_normal((B, H, NB, NB)).astype(np.float32)
+    s = np.round(rng.standard_normal((B, N)) * 50).astype(np.float32) / 50      # many exact ties
+    n_protect, k_keep = 3001, 40
+    idx, cnt, ptok, pblk = orc.build_block_mask(bs, s, n_protect, k_keep, blk, N)
+    out = av.avsa_build_block_mask(None, None, torch.from_numpy(s).cuda(), n_protect, k_keep, blk,
+                                   flags=av.AVSA_PROTECT_ROWS | av.AVSA_USE_GIVEN_BLOCK_SCORES,
+                                   block_scores=torch.from_numpy(bs).cuda(), shape=(B, H, N, d))
+    _status_ok(out["ws"])
+    assert np.array_equal(out["prot_tok"].cpu().numpy(), ptok)
+    assert np.array_equal(out["prot_blk"].cpu().numpy(), pblk)
+    assert np.array_equal(out["col_cnt"].cpu().numpy(), cnt)
+    assert np.array_equal(out["col_idx"].cpu().numpy(), idx)
+
+
 @pytest.mark.parametrize("name", ["tiny", "small128", "medium128"])
 def test_block_scores_and_selection_from_pooled_qk(name):
     w = wl.WORKLOADS[name]
