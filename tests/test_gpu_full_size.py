@@ -1,0 +1,105 @@
+"""Parity at the full Ovi-class size, in the launch configuration the benchmark times.
+
+The oracle cannot compute a whole layer in seconds, so: the mask is compared in full (bit-exact given the
+same fp32 score tensors), the cross-attention on a sample of heads, and the sparse attention on sampled
+query blocks (first, ragged last, protected and unprotected ones) at full key length -- rows of Eq. 10 are
+independent, so any subset can be checked alone.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import avsa_oracle as orc
+from paper_2608_15522_b200 import binding as av
+from paper_2608_15522_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+MAX_ABS = 1e-2
+REL_L2 = 5e-3
+
+
+def _np64(x):
+    return x.detach().double().cpu().numpy()
+
+
+def _close(got, want, what):
+    err = (np.abs(got - want) / np.maximum(1.0, np.abs(want))).max()
+    rel = np.linalg.norm((got - want).ravel()) / max(np.linalg.norm(want.ravel()), 1e-30)
+    assert np.isfinite(got).all(), what
+    assert err <= MAX_ABS and rel <= REL_L2, f"{what}: max-abs(scaled) {err:.3e}, rel-L2 {rel:.3e}"
+
+
+@pytest.fixture(scope="module")
+def ovi():
+    w = wl.WORKLOADS["ovi"]
+    dev = torch.device("cuda", 0)
+    q, k, v = wl.make_self_qkv(w, 0, dev)
+    qa, kc, vc = wl.make_cross_qkv(w, 0, dev)
+    return w, (q, k, v), (qa, kc, vc)
+
+
+def test_ovi_cross_attention_sampled_heads(ovi):
+    w, _, (qa, kc, vc) = ovi
+    gamma = 1.0 / (w.H * w.n_audio)
+    o, lse, s, ws = av.avsa_cross_attn_scores(qa, kc, vc, score_gamma=gamma)
+    assert av.avsa_read_status(ws)[0] == av.AVSA_OK
+    assert abs(float(s.sum()) - 1.0) < 2e-3
+    for h in (0, 11, 23):
+        want_o, want_lse, _ = orc.cross_attention(_np64(qa[:, h:h + 1]), _np64(kc[:, h:h + 1]), _np64(vc[:, h:h + 1]))
+        _close(_np64(o[:, h:h + 1]), want_o, f"cross O head {h}")
+        _close(_np64(lse[:, h:h + 1]), want_lse, f"cross lse head {h}")
+    # scores need every head: accumulate the oracle head by head (Eq. 2)
+    want_s = np.zeros((w.B, w.n_video))
+    for h in range(w.H):
+        _, _, A = orc.cross_attention(_np64(qa[:, h:h + 1]), _np64(kc[:, h:h + 1]), _np64(vc[:, h:h + 1]))
+        want_s = orc.column_scores(A, s_prev=want_s, beta=1.0, gamma=gamma)
+    got_s = _np64(s)
+    assert np.linalg.norm(got_s - want_s) / np.linalg.norm(want_s) <= REL_L2
+    assert np.abs(got_s - want_s).max() <= MAX_ABS
+    # most of the response mass sits in the planted regions, and so does the protected set
+    region = wl.region_mask(w, "cpu").numpy()
+    top = orc.topk_indices(want_s[0], orc.ceil_pct(w.protect_pct, w.n_video))
+    assert region[top].mean() > 0.9
+
+
+def test_ovi_mask_full_and_sparse_attention_sampled_blocks(ovi):
+    w, (q, k, v), (qa, kc, vc) = ovi
+    NB = w.n_blocks
+    n_protect = av.avsa_count_from_percent(w.protect_pct, w.n_video)
+    k_keep = av.avsa_count_from_percent(w.keep_pct, NB)
+    assert (n_protect, k_keep, NB) == (1638, 64, 256)
+    _, _, s, _ = av.avsa_cross_attn_scores(qa, kc, vc, score_gamma=1.0 / (w.H * w.n_audio))
+    m = av.avsa_build_block_mask(q, k, s, n_protect, k_keep, w.blk)
+    assert av.avsa_read_status(m["ws"])[0] == av.AVSA_OK
+    # block scores against the oracle (fp32 vs fp64), head by head to bound memory
+    bs_gpu = m["block_scores"].cpu().numpy()
+    for h in (0, 7, 23):
+        want = orc.block_scores(_np64(q[:, h:h + 1]), _np64(k[:, h:h + 1]), w.blk)
+        assert np.abs(bs_gpu[:, h:h + 1] - want).max() <= 1e-4 * max(1.0, np.abs(want).max())
+    # lists: the oracle selecting from the same fp32 tensors must agree bit for bit, everywhere
+    idx, cnt, ptok, pblk = orc.build_block_mask(bs_gpu, s.cpu().numpy(), n_protect, k_keep, w.blk, w.n_video)
+    assert np.array_equal(m["prot_tok"].cpu().numpy(), ptok)
+    assert np.array_equal(m["prot_blk"].cpu().numpy(), pblk)
+    assert np.array_equal(m["col_cnt"].cpu().numpy(), cnt)
+    assert np.array_equal(m["col_idx"].cpu().numpy(), idx)
+    assert ptok.sum() == n_protect and 0 < pblk.sum() < NB
+    # executed fraction vs Eq. 16's kappa + rho and its block-lifted form
+    pairs = cnt.sum() / float(w.H * NB * NB)
+    p_b = pblk.mean()
+    assert abs(pairs - (0.25 + p_b * 0.75)) < 1e-9 and pairs >= 0.25 + 0.05 - 1e-9
+    # sparse attention on sampled query blocks at full key length
+    o, lse, ws = av.avsa_sparse_self_attn(q, k, v, m["col_idx"], m["col_cnt"], w.blk, want_lse=True)
+    assert av.avsa_read_status(ws)[0] == av.AVSA_OK
+    rng = np.random.default_rng(0)
+    prot = np.nonzero(pblk[0])[0]
+    unprot = np.nonzero(pblk[0] == 0)[0]
+    blocks = [0, NB - 1] + rng.choice(prot, 3, replace=False).tolist() + rng.choice(unprot, 3, replace=False).tolist()
+    for h in (0, 13, 23):
+        kh, vh = _np64(k[0, h]), _np64(v[0, h])
+        for i in blocks:
+            lo, hi = i * w.blk, min((i + 1) * w.blk, w.n_video)
+            cols = [int(c) for c in idx[0, h, i, : cnt[0, h, i]]]
+            want_o, want_l = orc.masked_attention_rows(_np64(q[0, h, lo:hi]), kh, vh, cols, w.blk)
+            _close(_np64(o[0, h, lo:hi]), want_o, f"O head {h} block {i}")
+            _close(_np64(lse[0, h, lo:hi]), want_l, f"lse head {h} block {i}")
