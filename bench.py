@@ -258,11 +258,22 @@ def run_ours(args, w):
         b.record(); torch.cuda.synchronize()
         return a.elapsed_time(b) / n
 
+    # ---- token-exact protection (Eq. 9 on tokens): base-pattern lists + dense recomputation of protected rows
+    m_tok = av.avsa_build_block_mask(q, k, s, n_protect, k_keep, w.blk, flags=av.AVSA_PROTECT_TOKENS)
+    o_tok, _, ws_tok = av.avsa_sparse_self_attn(q, k, v, m_tok["col_idx"], m_tok["col_cnt"], w.blk)
+    ws_rows = av.avsa_protected_rows_attn(q, k, v, m_tok["prot_tok"], n_protect, w.blk, o_tok)
+    pairs_tok = int(m_tok["col_cnt"].sum().item())
+
+    def token_exact_attn():
+        av.avsa_sparse_self_attn(q, k, v, m_tok["col_idx"], m_tok["col_cnt"], w.blk, o=o_tok, ws=ws_tok)
+        av.avsa_protected_rows_attn(q, k, v, m_tok["prot_tok"], n_protect, w.blk, o_tok, ws=ws_rows)
+
     t_dense_ours = time_fn(lambda: av.avsa_sparse_self_attn(q, k, v, idx_all, cnt_all, w.blk, o=o, ws=ws3), 3)
     try:
         t_dense_lib = time_fn(lambda: torch.nn.functional.scaled_dot_product_attention(q, k, v), 3)
     except Exception:
         t_dense_lib = None
+    t_token_exact = time_fn(token_exact_attn, 5)
     del idx_all, cnt_all
 
     # ---- end to end through the public API with host buffers (pinned), copies inside the timed region
@@ -326,6 +337,15 @@ def run_ours(args, w):
                    "dense_keep_all_ours": t_dense_ours, "dense_library_sdpa": t_dense_lib},
             "speedup_vs_dense": {"attn_only": dense_best / t_attn, "layer_step": dense_best / ms_per_step,
                                  "dense_is": "library_sdpa" if dense_best == t_dense_lib else "keep_all_ours"},
+            "token_exact_protection": {
+                "note": "Eq. 9 on tokens: base-pattern lists (avsa_build_block_mask with AVSA_PROTECT_TOKENS) + "
+                        "avsa_sparse_self_attn + avsa_protected_rows_attn; timed outside the step loop",
+                "attn_ms": t_token_exact,
+                "executed_fraction": (pairs_tok * w.blk * w.blk + w.B * w.H * n_protect * float(w.n_video))
+                                     / (w.B * w.H * float(w.n_video) ** 2),
+                "kappa_plus_rho": (w.keep_pct + w.protect_pct) / 100.0,
+                "speedup_vs_dense": dense_best / t_token_exact,
+                "dense_equiv_tflops": fl_dense / (t_token_exact * 1e-3) / 1e12},
             "executed_tflops": achieved,
             "roofline": {"kernel": "attn_fwd_kernel<128,128,MODE_LIST> (avsa_sparse_self_attn)", "bound": "tensor",
                          "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,

@@ -61,6 +61,8 @@ typedef struct {
 #define AVSA_PROTECT_ROWS 1u            /* Eq. 9: a protected query block keeps every key block */
 #define AVSA_PROTECT_COLS 2u            /* opt-in superset: protected key blocks visible to all rows */
 #define AVSA_USE_GIVEN_BLOCK_SCORES 4u  /* block_scores is an input; q and k are not read */
+#define AVSA_PROTECT_TOKENS 8u          /* lists carry the base pattern only (no block is made dense); the
+                                           protected rows are restored by avsa_protected_rows_attn */
 
 /*
  * (1) Cross-attention with response scores -- Eq. 1, Eq. 2 (and the running blend of Eq. 4).
@@ -100,7 +102,7 @@ AVSA_API size_t avsa_cross_attn_scores_workspace_bytes(int B, int H, int Nq, int
  *
  * Every top-k orders by (value larger, then index smaller); NaN ranks as -inf; -0 equals +0.
  * Given the same fp32 scores / block_scores the outputs are exactly determined (integer results).
- * flags == 0 is treated as AVSA_PROTECT_ROWS.  NB <= 2048.
+ * Without any AVSA_PROTECT_* flag AVSA_PROTECT_ROWS is assumed.  NB <= 2048.
  */
 AVSA_API int avsa_build_block_mask(int B, int H, int N, int d, int blk, avsa_bf16_4d q, avsa_bf16_4d k, const float* scores,
                           int n_protect, int k_keep, unsigned flags, float softmax_scale, float* block_scores,
@@ -122,6 +124,24 @@ AVSA_API int avsa_sparse_self_attn(int B, int H, int N, int d, int blk, avsa_bf1
                           const int32_t* col_idx, const int32_t* col_cnt, void* o_bf16, float* lse,
                           float softmax_scale, void* ws, size_t ws_bytes, void* stream);
 AVSA_API size_t avsa_sparse_self_attn_workspace_bytes(int B, int H, int N, int d, int blk);
+
+/*
+ * (4) Token-exact protection -- Eq. 9 applied to tokens, i.e. the row-wise form of Eq. 11: the rows of
+ * the protected tokens are dense attention rows ("dense-row recomputation" in the paper's notes).
+ *
+ * Use with lists built under AVSA_PROTECT_TOKENS: run avsa_sparse_self_attn first, then this call, which
+ * recomputes o[b,h,i,:] (and lse[b,h,i], if given) for every token i with prot_tok[b,i] != 0 as dense
+ * attention over all N keys and overwrites those rows in place.  The cost is n_protect * N per head
+ * (Eq. 16's rho N^2 term) instead of a whole block row per touched block.
+ *   prot_tok   uint8 [B,N] as written by avsa_build_block_mask; exactly n_protect flags per batch item,
+ *              otherwise AVSA_ERR_BAD_MASK is recorded and that batch item is left untouched
+ *   o_bf16     in/out, bf16 with the strides of q;  lse in/out fp32 [B,H,N] or NULL
+ * n_protect == 0 is a no-op.  The workspace also depends on n_protect.
+ */
+AVSA_API int avsa_protected_rows_attn(int B, int H, int N, int d, int blk, avsa_bf16_4d q, avsa_bf16_4d k,
+                                      avsa_bf16_4d v, const uint8_t* prot_tok, int n_protect, void* o_bf16,
+                                      float* lse, float softmax_scale, void* ws, size_t ws_bytes, void* stream);
+AVSA_API size_t avsa_protected_rows_attn_workspace_bytes(int B, int H, int N, int d, int blk, int n_protect);
 
 /*
  * Allocation-free variant of avsa_build_block_mask.  The paper has no counterpart; this is a

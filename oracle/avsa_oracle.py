@@ -14,6 +14,7 @@ What follows the paper and what is this build's reading of it:
   leaves S_m to "a standard sparse-attention method"; the rule here (mean-pooled Q/K block scores,
   per-head top-k) is this build's choice.  PARITY UNPINNED against the paper's own system for this
   rule; the functions are pinned against brute force and closed forms only.
+* ``protected_attention_token_exact``               -- Eq. 9 / Eq. 11 on tokens (dense rows for protected tokens).
 * ``protected_blocks``, ``build_block_mask``       -- Eq. 9 lifted from tokens to blocks: a block is
   protected iff it holds at least one protected token (a superset of the token-level rule).
 
@@ -222,6 +223,27 @@ def masked_attention(q, k, v, col_idx, col_cnt, blk, scale=None):
                 cols = [int(c) for c in col_idx[b, h, i, : int(col_cnt[b, h, i])]]
                 out[b, h, lo:hi], lse[b, h, lo:hi] = masked_attention_rows(
                     q[b, h, lo:hi], k[b, h], v[b, h], cols, blk, scale)
+    return out, lse
+
+
+def protected_attention_token_exact(q, k, v, col_idx, col_cnt, prot_tok, blk, scale=None):
+    """Eq. 11 read on tokens: rows of protected tokens are dense attention rows (Eq. 5), every other row
+    follows the sparse pattern given by the lists (Eq. 7).  The lists hold the base pattern only.
+    q,k,v [B,H,N,d]; prot_tok [B,N] -> (O [B,H,N,d], lse [B,H,N])."""
+    q = np.asarray(q, np.float64); k = np.asarray(k, np.float64); v = np.asarray(v, np.float64)
+    out, lse = masked_attention(q, k, v, col_idx, col_cnt, blk, scale)
+    B, H, N, d = q.shape
+    for b in range(B):
+        rows = np.nonzero(np.asarray(prot_tok)[b])[0]
+        if len(rows) == 0:
+            continue
+        for h in range(H):
+            s = (q[b, h, rows] @ k[b, h].T) * _scale(d, scale)
+            m = s.max(axis=1, keepdims=True)
+            e = np.exp(s - m)
+            l = e.sum(axis=1, keepdims=True)
+            out[b, h, rows] = (e / l) @ v[b, h]
+            lse[b, h, rows] = (m + np.log(l))[:, 0]
     return out, lse
 
 

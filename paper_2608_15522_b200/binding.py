@@ -26,11 +26,13 @@ AVSA_ERR_BAD_MASK = 6
 AVSA_PROTECT_ROWS = 1
 AVSA_PROTECT_COLS = 2
 AVSA_USE_GIVEN_BLOCK_SCORES = 4
+AVSA_PROTECT_TOKENS = 8
 
 EXPORTS = (
     "avsa_cross_attn_scores", "avsa_cross_attn_scores_workspace_bytes",
     "avsa_build_block_mask", "avsa_build_block_mask_workspace_bytes", "avsa_build_block_mask_static",
     "avsa_sparse_self_attn", "avsa_sparse_self_attn_workspace_bytes",
+    "avsa_protected_rows_attn", "avsa_protected_rows_attn_workspace_bytes",
     "avsa_count_from_percent", "avsa_read_status", "avsa_status_string", "avsa_version",
 )
 
@@ -74,6 +76,10 @@ def load_library() -> ctypes.CDLL:
     lib.avsa_sparse_self_attn.restype = i
     lib.avsa_sparse_self_attn_workspace_bytes.argtypes = [i, i, i, i, i]
     lib.avsa_sparse_self_attn_workspace_bytes.restype = sz
+    lib.avsa_protected_rows_attn.argtypes = [i, i, i, i, i, T, T, T, vp, i, vp, vp, f, vp, sz, vp]
+    lib.avsa_protected_rows_attn.restype = i
+    lib.avsa_protected_rows_attn_workspace_bytes.argtypes = [i, i, i, i, i, i]
+    lib.avsa_protected_rows_attn_workspace_bytes.restype = sz
     lib.avsa_count_from_percent.argtypes = [i, i]
     lib.avsa_count_from_percent.restype = i
     lib.avsa_read_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_int)]
@@ -253,3 +259,20 @@ def avsa_sparse_self_attn(q, k, v, col_idx, col_cnt, blk, softmax_scale=0.0, wan
                                    _ptr(lse), float(softmax_scale), _ptr(ws), ws.numel(), _stream(dev))
     _check(st, "avsa_sparse_self_attn")
     return o, lse, ws
+
+
+def avsa_protected_rows_attn_workspace_bytes(B, H, N, d, blk, n_protect) -> int:
+    return int(load_library().avsa_protected_rows_attn_workspace_bytes(B, H, N, d, blk, n_protect))
+
+
+def avsa_protected_rows_attn(q, k, v, prot_tok, n_protect, blk, o, lse=None, softmax_scale=0.0, ws=None):
+    """Eq. 9 / Eq. 11 on tokens: overwrites the rows of the protected tokens in ``o`` (and ``lse``) with dense
+    attention rows.  Returns ws."""
+    lib = load_library()
+    B, H, N, d = q.shape
+    dev = q.device
+    ws = _workspace(avsa_protected_rows_attn_workspace_bytes(B, H, N, d, blk, int(n_protect)), dev, ws)
+    st = lib.avsa_protected_rows_attn(B, H, N, d, blk, _t4(q), _t4(k), _t4(v), _ptr(prot_tok), int(n_protect), _ptr(o),
+                                      _ptr(lse), float(softmax_scale), _ptr(ws), ws.numel(), _stream(dev))
+    _check(st, "avsa_protected_rows_attn")
+    return ws

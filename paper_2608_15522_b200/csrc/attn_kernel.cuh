@@ -400,4 +400,53 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__
   if (warp == 2) tmem_dealloc(tmem, 512);
 }
 
+// ------------------------------------------------------------------------------------------------
+// Merge of the key-axis splits written by MODE_RANGE: for every query row, combine the normalised
+// partial outputs with weights exp2(lse2_split - max) and write bf16 rows and the natural-log LSE.
+// With a row map the result of compact row r goes to row row_map[b][r] of the output (rows mapped to
+// a negative index are skipped): that is how recomputed protected rows are scattered back.
+// ------------------------------------------------------------------------------------------------
+template <int BLK, int D>
+__global__ void __launch_bounds__(128) merge_splits_kernel(const float* __restrict__ part_o,
+                                                           const float* __restrict__ part_lse2, int n_split, int NQT,
+                                                           int Nq, int H, int total_rows, __nv_bfloat16* __restrict__ o,
+                                                           int64_t o_sb, int64_t o_sh, int64_t o_sn,
+                                                           float* __restrict__ lse, const int32_t* __restrict__ row_map,
+                                                           int row_map_stride, int n_out) {
+  constexpr int TPR = D / 4;
+  const int rg = blockIdx.x * (128 / TPR) + threadIdx.x / TPR;
+  const int c4 = threadIdx.x % TPR;
+  if (rg >= total_rows) return;
+  const int bh = rg / Nq, qrow = rg % Nq;
+  const int b = bh / H, h = bh % H;
+  int out_row = qrow;
+  if (row_map != nullptr) {
+    out_row = row_map[static_cast<int64_t>(b) * row_map_stride + qrow];
+    if (out_row < 0 || out_row >= n_out) return;
+  }
+  const int qt = qrow / BLK, r = qrow % BLK;
+  const int64_t item0 = (static_cast<int64_t>(bh) * NQT + qt) * n_split;
+  float M = -INFINITY;
+  for (int s = 0; s < n_split; s++) M = fmaxf(M, part_lse2[(item0 + s) * BLK + r]);
+  float W = 0.f;
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int s = 0; s < n_split; s++) {
+    const float w = exp2f(part_lse2[(item0 + s) * BLK + r] - M);
+    const float4 v = *reinterpret_cast<const float4*>(part_o + ((item0 + s) * BLK + r) * D + c4 * 4);
+    W += w;
+    acc.x = fmaf(w, v.x, acc.x);
+    acc.y = fmaf(w, v.y, acc.y);
+    acc.z = fmaf(w, v.z, acc.z);
+    acc.w = fmaf(w, v.w, acc.w);
+  }
+  const float inv = 1.0f / W;
+  if (o != nullptr) {
+    uint2 pk;
+    pk.x = pack_bf16x2(acc.x * inv, acc.y * inv);
+    pk.y = pack_bf16x2(acc.z * inv, acc.w * inv);
+    *reinterpret_cast<uint2*>(o + b * o_sb + h * o_sh + out_row * o_sn + c4 * 4) = pk;
+  }
+  if (c4 == 0 && lse != nullptr) lse[static_cast<int64_t>(bh) * n_out + out_row] = (M + log2f(W)) * 0.6931471805599453f;
+}
+
 }  // namespace avsa

@@ -8,46 +8,6 @@
 namespace avsa {
 
 // ------------------------------------------------------------------------------------------------
-// pass 1 merge: combine the splits of the key axis of every query row
-// ------------------------------------------------------------------------------------------------
-template <int BLK, int D>
-__global__ void __launch_bounds__(128) merge_splits_kernel(const float* __restrict__ part_o,
-                                                           const float* __restrict__ part_lse2, int n_split, int NQT,
-                                                           int Nq, int H, int total_rows, __nv_bfloat16* __restrict__ o,
-                                                           int64_t o_sb, int64_t o_sh, int64_t o_sn,
-                                                           float* __restrict__ lse) {
-  constexpr int TPR = D / 4;
-  const int rg = blockIdx.x * (128 / TPR) + threadIdx.x / TPR;
-  const int c4 = threadIdx.x % TPR;
-  if (rg >= total_rows) return;
-  const int bh = rg / Nq, qrow = rg % Nq;
-  const int qt = qrow / BLK, r = qrow % BLK;
-  const int64_t item0 = (static_cast<int64_t>(bh) * NQT + qt) * n_split;
-  float M = -INFINITY;
-  for (int s = 0; s < n_split; s++) M = fmaxf(M, part_lse2[(item0 + s) * BLK + r]);
-  float W = 0.f;
-  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-  for (int s = 0; s < n_split; s++) {
-    const float w = exp2f(part_lse2[(item0 + s) * BLK + r] - M);
-    const float4 v = *reinterpret_cast<const float4*>(part_o + ((item0 + s) * BLK + r) * D + c4 * 4);
-    W += w;
-    acc.x = fmaf(w, v.x, acc.x);
-    acc.y = fmaf(w, v.y, acc.y);
-    acc.z = fmaf(w, v.z, acc.z);
-    acc.w = fmaf(w, v.w, acc.w);
-  }
-  const float inv = 1.0f / W;
-  if (o != nullptr) {
-    const int b = bh / H, h = bh % H;
-    uint2 pk;
-    pk.x = pack_bf16x2(acc.x * inv, acc.y * inv);
-    pk.y = pack_bf16x2(acc.z * inv, acc.w * inv);
-    *reinterpret_cast<uint2*>(o + b * o_sb + h * o_sh + qrow * o_sn + c4 * 4) = pk;
-  }
-  if (c4 == 0) lse[rg] = (M + log2f(W)) * 0.6931471805599453f;
-}
-
-// ------------------------------------------------------------------------------------------------
 // pass 2: column sums of the attention map.  One CTA keeps the queries of one (batch, head) in
 // shared memory and walks a range of 128-key tiles.  S^T[key, query] accumulates in tensor memory
 // (two buffers of up to 256 columns); two groups of 128 threads (one thread per key row) turn
@@ -266,8 +226,8 @@ static CrossPlan make_cross_plan(int B, int H, int Nq, int Nk, int d) {
   c.blk = d;   // (blk, d) = (128,128) or (64,64)
   c.NQT = (Nq + c.blk - 1) / c.blk;
   c.NKB = (Nk + c.blk - 1) / c.blk;
-  const int target = 296;   // about two CTAs per SM's worth of work items
-  int want_split = (target + B * H * c.NQT - 1) / (B * H * c.NQT);
+  const int target = 296;   // two work items per SM (148 SMs, one CTA each): whole waves, no ragged third one
+  int want_split = target / (B * H * c.NQT);
   if (want_split < 1) want_split = 1;
   if (want_split > c.NKB) want_split = c.NKB;
   c.tps = (c.NKB + want_split - 1) / want_split;
@@ -275,7 +235,7 @@ static CrossPlan make_cross_plan(int B, int H, int Nq, int Nk, int d) {
   c.NKT = (Nk + 127) / 128;
   c.NCH = Nq > 256 ? 2 : 1;
   c.W = (((Nq + c.NCH - 1) / c.NCH) + 15) / 16 * 16;
-  int want_range = (target + B * H - 1) / (B * H);
+  int want_range = target / (B * H);
   if (want_range < 1) want_range = 1;
   if (want_range > c.NKT) want_range = c.NKT;
   c.tpr = (c.NKT + want_range - 1) / want_range;
@@ -328,7 +288,7 @@ static int run_cross(int B, int H, int Nq, int Nk, const avsa_bf16_4d& q, const 
     constexpr int RPB = 128 / (D / 4);
     merge_splits_kernel<BLK, D><<<(total_rows + RPB - 1) / RPB, 128, 0, st>>>(
         part_o, part_lse, c.n_split, c.NQT, Nq, H, total_rows, static_cast<__nv_bfloat16*>(o), q.stride_b, q.stride_h,
-        q.stride_n, lse);
+        q.stride_n, lse, nullptr, 0, Nq);
   }
   // ---- pass 2
   if (scores != nullptr) {

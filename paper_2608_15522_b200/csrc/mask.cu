@@ -426,7 +426,7 @@ extern "C" int avsa_build_block_mask(int B, int H, int N, int d, int blk, avsa_b
   if (n_protect > 0 && scores == nullptr) return AVSA_ERR_INVALID_ARG;
   const bool given = (flags & AVSA_USE_GIVEN_BLOCK_SCORES) != 0;
   if (!given && (!tensor_ok(q, B, H) || !tensor_ok(k, B, H))) return AVSA_ERR_INVALID_ARG;
-  if ((flags & (AVSA_PROTECT_ROWS | AVSA_PROTECT_COLS)) == 0) flags |= AVSA_PROTECT_ROWS;
+  if ((flags & (AVSA_PROTECT_ROWS | AVSA_PROTECT_COLS | AVSA_PROTECT_TOKENS)) == 0) flags |= AVSA_PROTECT_ROWS;
   const MaskWorkspace w = mask_ws_layout(B, H, N, d, blk);
   if (ws == nullptr || ws_bytes < w.total) return AVSA_ERR_WORKSPACE;
   cudaStream_t st = as_stream(stream);

@@ -305,6 +305,43 @@ def test_whole_path_tiny_matches_oracle():
     _close(_np64(o), want, "whole path O")
 
 
+# ------------------------------------------------------------------------------------------- token-exact protection
+@pytest.mark.parametrize("name", ["tiny", "small128", "medium128"])
+def test_token_exact_protection_matches_oracle(name):
+    w = wl.WORKLOADS[name]
+    q, k, v = wl.make_self_qkv(w, 6)
+    _, _, _, s64 = _oracle_scores(w, 6)
+    n_protect = orc.ceil_pct(w.protect_pct, w.n_video)
+    k_keep = max(1, orc.ceil_pct(w.keep_pct, w.n_blocks))
+    bs32 = orc.block_scores(_np64(q), _np64(k), w.blk).astype(np.float32)
+    s32 = s64.astype(np.float32)
+    idx, cnt, ptok, _ = orc.build_block_mask(bs32, s32, n_protect, k_keep, w.blk, w.n_video, protect_rows=False)
+    m = av.avsa_build_block_mask(None, None, torch.from_numpy(s32).cuda(), n_protect, k_keep, w.blk,
+                                 flags=av.AVSA_PROTECT_TOKENS | av.AVSA_USE_GIVEN_BLOCK_SCORES,
+                                 block_scores=torch.from_numpy(bs32).cuda(), shape=(w.B, w.H, w.n_video, w.d))
+    assert np.array_equal(m["col_idx"].cpu().numpy(), idx) and np.array_equal(m["col_cnt"].cpu().numpy(), cnt)
+    assert np.array_equal(m["prot_tok"].cpu().numpy(), ptok)
+    assert (cnt == k_keep).all()                                       # no block is made dense
+    qc, kc, vc = q.cuda(), k.cuda(), v.cuda()
+    o, lse, ws = av.avsa_sparse_self_attn(qc, kc, vc, m["col_idx"], m["col_cnt"], w.blk, want_lse=True)
+    _status_ok(ws)
+    ws2 = av.avsa_protected_rows_attn(qc, kc, vc, m["prot_tok"], n_protect, w.blk, o, lse=lse)
+    _status_ok(ws2)
+    want_o, want_l = orc.protected_attention_token_exact(_np64(q), _np64(k), _np64(v), idx, cnt, ptok, w.blk)
+    _close(_np64(o), want_o, f"{name} token-exact O")
+    _close(_np64(lse), want_l, f"{name} token-exact lse")
+    # a flag count that disagrees with n_protect is refused on the device and nothing is overwritten
+    before = o.clone()
+    ws3 = av.avsa_protected_rows_attn(qc, kc, vc, m["prot_tok"], n_protect + 1, w.blk, o)
+    code, detail = av.avsa_read_status(ws3)
+    assert code == av.AVSA_ERR_BAD_MASK and detail[2] == n_protect
+    assert torch.equal(before, o)
+    # zero protected tokens: a no-op
+    av.avsa_protected_rows_attn(qc, kc, vc, torch.zeros_like(m["prot_tok"]), 0, w.blk, o)
+    torch.cuda.synchronize()
+    assert torch.equal(before, o)
+
+
 def test_host_side_argument_errors():
     w = wl.WORKLOADS["tiny"]
     q, k, v = (t.cuda() for t in wl.make_self_qkv(w, 0))

@@ -327,3 +327,31 @@ def test_masked_attention_brute_force_single_row():
             want = sum(math.exp(x) / z * v[j, t] for x, j in zip(logits, keys))
             assert abs(o[r, t] - want) < 1e-13
         assert abs(lse[r] - math.log(z)) < 1e-13
+
+
+def test_token_exact_protection_is_eq9_on_tokens():
+    """Eq. 9 written literally on tokens: 0 where the query is protected or the pair is in S, -inf elsewhere."""
+    B, H, N, d, blk = 1, 2, 45, 8, 8
+    q, k, v = _rand((B, H, N, d), 31), _rand((B, H, N, d), 32), _rand((B, H, N, d), 33)
+    bs = orc.block_scores(q, k, blk)
+    s = _rand((B, N), 34)
+    n_protect = 4
+    idx, cnt, ptok, pblk = orc.build_block_mask(bs, s, n_protect, 2, blk, N, protect_rows=False)
+    assert (cnt == 2).all()                                            # base pattern only
+    O, lse = orc.protected_attention_token_exact(q, k, v, idx, cnt, ptok, blk)
+    dense, dense_lse = orc.dense_attention(q, k, v)
+    sparse, _ = orc.masked_attention(q, k, v, idx, cnt, blk)
+    for h in range(H):
+        M = np.full((N, N), -np.inf)
+        for i in range(6):
+            for j in idx[0, h, i, : cnt[0, h, i]]:
+                M[i * blk:(i + 1) * blk, j * blk:(j + 1) * blk] = 0.0
+        M[ptok[0] == 1, :] = 0.0
+        logits = q[0, h] @ k[0, h].T / math.sqrt(d) + M
+        want = torch.softmax(torch.from_numpy(logits), dim=-1).numpy() @ v[0, h]
+        np.testing.assert_allclose(O[0, h], want, rtol=1e-11, atol=1e-12)
+        prot = ptok[0] == 1
+        np.testing.assert_allclose(O[0, h, prot], dense[0, h, prot], rtol=1e-12, atol=1e-13)      # Eq. 11, first case
+        np.testing.assert_allclose(lse[0, h, prot], dense_lse[0, h, prot], rtol=1e-12)
+        np.testing.assert_allclose(O[0, h, ~prot], sparse[0, h, ~prot], rtol=1e-12, atol=1e-13)   # Eq. 11, second case
+    assert ptok.sum() == n_protect
