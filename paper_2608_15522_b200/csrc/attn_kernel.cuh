@@ -40,7 +40,7 @@ struct AttnSmem {
   static constexpr int kK = kQBytes;
   static constexpr int kV = kK + kStages * kTileBytes;
   static constexpr int kBars = kV + kStages * kTileBytes;
-  static constexpr int kNumBars = 1 + 4 * kStages + 2 + 2 + 1;
+  static constexpr int kNumBars = 1 + 4 * kStages + 2 + 4 + 1;
   static constexpr int kStats = kBars + kNumBars * 8;          // float [2][2][128]: m, l per group and row
   static constexpr int kMisc = kStats + 2 * 2 * 128 * 4;       // tmem base, abort flag
   static constexpr int kTotal = kMisc + 16;
@@ -61,7 +61,20 @@ struct AttnParams {
   int Nq, NQT;              // query rows and query tiles
   int Nk, NKB;              // key rows and key tiles
   float scale_log2;         // softmax_scale * log2(e)
+#ifdef AVSA_TRACE
+  long long* trace;         // [3 roles][64 tiles][8 stamps] clock64 stamps of CTA (0,0,0), for pipeline analysis
+#endif
 };
+
+#ifdef AVSA_TRACE
+#define AVSA_STAMP(role, tile, slot)                                                                    \
+  do {                                                                                                  \
+    if (p.trace != nullptr && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && (tile) < 64)     \
+      p.trace[((role) * 64 + (tile)) * 8 + (slot)] = clock64();                                         \
+  } while (0)
+#else
+#define AVSA_STAMP(role, tile, slot) do { } while (0)
+#endif
 
 template <int BLK, int D, int MODE>
 __global__ void __launch_bounds__(kAttnThreads, 1)
@@ -117,7 +130,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__
   const uint32_t bar0 = smem_u32(bars);
   auto BAR = [&](int i) { return bar0 + static_cast<uint32_t>(i) * 8u; };
   constexpr int Q_FULL = 0, K_FULL = 1, K_EMPTY = 1 + kStages, V_FULL = 1 + 2 * kStages, V_EMPTY = 1 + 3 * kStages,
-                S_FULL = 1 + 4 * kStages, P_FULL = S_FULL + 2, FINAL = P_FULL + 2;
+                S_FULL = 1 + 4 * kStages, P_FULL = S_FULL + 2, FINAL = P_FULL + 4;   // P_FULL + 2*group + half
   float* stats = reinterpret_cast<float*>(smem + L::kStats);
   volatile uint32_t* misc = reinterpret_cast<volatile uint32_t*>(smem + L::kMisc);   // [0] tmem base, [1] abort
 
@@ -131,7 +144,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__
     }
     for (int w = 0; w < 2; w++) {
       mbar_init(BAR(S_FULL + w), 1);
-      mbar_init(BAR(P_FULL + w), 128);
+      mbar_init(BAR(P_FULL + 2 * w), 128);
+      mbar_init(BAR(P_FULL + 2 * w + 1), 128);
     }
     mbar_init(BAR(FINAL), 1);
     misc[1] = 0u;
@@ -153,7 +167,10 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__
   const uint32_t TM_O[2] = {tmem + 256u, tmem + 384u};
 
   // A wait that gives up: records where, raises the CTA-wide abort flag, and lets every role unwind.
+  // The fast path is a single try_wait (the issuing thread's waits sit between MMA batches, so their
+  // latency shows up as tensor-pipe bubbles).
   auto wait_or_abort = [&](int bar, uint32_t parity, int where, int tile) -> bool {
+    if (mbar_try_wait(BAR(bar), parity)) return true;
     if (misc[1] != 0u) return false;
     if (mbar_wait(BAR(bar), parity)) return true;
     report_status(p.status, AVSA_ERR_TIMEOUT, where, item, tile);
@@ -203,44 +220,87 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     asm volatile("setmaxnreg.dec.sync.aligned.u32 64;");
-    if (lane == 0) {
-      const uint32_t idesc_qk = make_idesc_bf16(128, BLK, 0, 0);
-      const uint32_t idesc_pv = make_idesc_bf16(128, D, 0, 1);
-      const uint32_t q_addr = smem_u32(smem + L::kQ);
-      bool ok = wait_or_abort(Q_FULL, 0, kWhereQFull, 0);
+    {
+      // The whole warp runs this loop (uniform control flow keeps stage indices, addresses and descriptors in
+      // the uniform datapath); one elected lane issues the MMAs and commits.  The issuing lane must keep the
+      // tensor pipe's queue full (one MMA retires every 64 cycles), so per-MMA scalar work is kept minimal.
+      const bool leader = elect_one_sync();
+      constexpr uint32_t idesc_qk = make_idesc_bf16(128, BLK, 0, 0);
+      constexpr uint32_t idesc_pv = make_idesc_bf16(128, D, 0, 1);
+      constexpr uint32_t desc_hi = (1024u >> 4) | (1u << 14) | (2u << 29);            // SBO 1024 B, version, 128B swizzle
+      const uint32_t q_lo = ((smem_u32(smem + L::kQ) & 0x3FFFFu) >> 4) | (1u << 16);  // LBO field unused for K-major
+      const uint32_t k_lo0 = ((smem_u32(smem + L::kK) & 0x3FFFFu) >> 4) | (1u << 16);
+      const uint32_t v_lo0 = ((smem_u32(smem + L::kV) & 0x3FFFFu) >> 4) | (static_cast<uint32_t>(PANEL_BYTES >> 4) << 16);
+      const uint32_t tmem_u = __shfl_sync(0xffffffffu, tmem, 0);
+      auto desc64 = [](uint32_t lo) { return (static_cast<uint64_t>(desc_hi) << 32) | lo; };
+      auto wait_all = [&](int bar, uint32_t parity, int where, int tile) -> bool {
+        const bool r = wait_or_abort(bar, parity, where, tile);
+        return __all_sync(0xffffffffu, r);
+      };
+      bool ok = wait_all(Q_FULL, 0, kWhereQFull, 0);
+      int sk = 0, fk = 0;      // stage / fill parity of the tile whose S is issued
+      int sv = 0, fv = 0;      // same for the tile whose P V is issued
       for (int t = 0; t <= cnt && ok; t++) {
         if (t < cnt) {
-          const int w = t & 1, s = t % kStages, f = t / kStages;
-          ok = wait_or_abort(K_FULL + s, f & 1, kWhereKFull, t);
+          const int w = t & 1;
+          if (leader) AVSA_STAMP(0, t, 5);
+          ok = wait_all(K_FULL + sk, fk, kWhereKFull, t);
           if (!ok) break;
           tc_fence_after();
-          const uint32_t k_addr = smem_u32(smem + L::kK) + s * L::kTileBytes;
+          const uint32_t k_lo = k_lo0 + sk * (L::kTileBytes >> 4);
+          const uint32_t tm_s = tmem_u + (w << 7);
+          if (leader) {
+            AVSA_STAMP(0, t, 0);
 #pragma unroll
-          for (int ks = 0; ks < D / 16; ks++) {
-            const uint64_t ad = make_sdesc(q_addr + (ks >> 2) * QPANEL_BYTES + (ks & 3) * 32, 16, 1024);
-            const uint64_t bd = make_sdesc(k_addr + (ks >> 2) * PANEL_BYTES + (ks & 3) * 32, 16, 1024);
-            umma_ss(TM_S[w], ad, bd, idesc_qk, ks > 0 ? 1u : 0u);
+            for (int ks = 0; ks < D / 16; ks++) {
+              const uint32_t qoff = ((ks >> 2) * QPANEL_BYTES + (ks & 3) * 32) >> 4;
+              const uint32_t koff = ((ks >> 2) * PANEL_BYTES + (ks & 3) * 32) >> 4;
+              umma_ss(tm_s, desc64(q_lo + qoff), desc64(k_lo + koff), idesc_qk, ks > 0 ? 1u : 0u);
+            }
+            umma_commit(BAR(S_FULL + w));
+            umma_commit(BAR(K_EMPTY + sk));
+            AVSA_STAMP(0, t, 1);
           }
-          umma_commit(BAR(S_FULL + w));
-          umma_commit(BAR(K_EMPTY + s));
+          __syncwarp();
+          if (++sk == kStages) { sk = 0; fk ^= 1; }
         }
         if (t >= 1) {
-          const int u = t - 1, w = u & 1, s = u % kStages, f = u / kStages, i = u >> 1;
-          ok = wait_or_abort(P_FULL + w, i & 1, kWherePFull, u);
+          const int u = t - 1, w = u & 1, i = u >> 1;
+          if (leader) AVSA_STAMP(0, u, 2);
+          // P arrives in two halves of the key axis: the first half of the product starts while the
+          // softmax group is still exponentiating the second half
+          ok = wait_all(P_FULL + 2 * w, i & 1, kWherePFull, u);
           if (!ok) break;
-          ok = wait_or_abort(V_FULL + s, f & 1, kWhereVFull, u);
+          if (leader) AVSA_STAMP(0, u, 3);
+          ok = wait_all(V_FULL + sv, fv, kWhereVFull, u);
           if (!ok) break;
           tc_fence_after();
-          const uint32_t v_addr = smem_u32(smem + L::kV) + s * L::kTileBytes;
+          const uint32_t v_lo = v_lo0 + sv * (L::kTileBytes >> 4);
+          const uint32_t tm_p = tmem_u + (w << 7), tm_o = tmem_u + 256u + (w << 7);
+          const uint32_t acc0 = i > 0 ? 1u : 0u;
+          if (leader) {
+            AVSA_STAMP(0, u, 6);
 #pragma unroll
-          for (int ks = 0; ks < BLK / 16; ks++) {
-            const uint64_t bd = make_sdesc(v_addr + ks * 2048, PANEL_BYTES, 1024);
-            umma_ts(TM_O[w], TM_S[w] + ks * 8, bd, idesc_pv, (i > 0 || ks > 0) ? 1u : 0u);
+            for (int ks = 0; ks < BLK / 32; ks++)
+              umma_ts(tm_o, tm_p + ks * 8, desc64(v_lo + ks * (2048 >> 4)), idesc_pv, ks > 0 ? 1u : acc0);
           }
-          umma_commit(BAR(V_EMPTY + s));
+          __syncwarp();
+          ok = wait_all(P_FULL + 2 * w + 1, i & 1, kWherePFull, u);
+          if (!ok) break;
+          tc_fence_after();
+          if (leader) {
+#pragma unroll
+            for (int ks = BLK / 32; ks < BLK / 16; ks++)
+              umma_ts(tm_o, tm_p + ks * 8, desc64(v_lo + ks * (2048 >> 4)), idesc_pv, 1u);
+            umma_commit(BAR(V_EMPTY + sv));
+            AVSA_STAMP(0, u, 4);
+          }
+          __syncwarp();
+          if (++sv == kStages) { sv = 0; fv ^= 1; }
         }
       }
-      if (ok) umma_commit(BAR(FINAL));
+      if (ok && leader) umma_commit(BAR(FINAL));
+      __syncwarp();
     }
   } else if (warp < 4) {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 64;");
@@ -257,14 +317,17 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__
     bool ok = true;
     for (int i = 0; i < nw && ok; i++) {
       const int t = 2 * i + w;
+      if ((warp & 3) == 0 && lane == 0) AVSA_STAMP(1 + w, t, 0);
       ok = wait_or_abort(S_FULL + w, i & 1, kWhereSFull, t);
       if (!ok) break;
       tc_fence_after();
+      if ((warp & 3) == 0 && lane == 0) AVSA_STAMP(1 + w, t, 1);
       uint32_t s[BLK];
 #pragma unroll
       for (int c = 0; c < BLK / 32; c++)
         tmem_ld32(TM_S[w] + lane_off + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
       tmem_wait_ld();
+      if ((warp & 3) == 0 && lane == 0) AVSA_STAMP(1 + w, t, 2);
       if (t == cnt - 1 && ragged_valid < BLK) {
 #pragma unroll
         for (int j = 0; j < BLK; j++)
@@ -298,6 +361,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__
         }
       }
       l_run *= factor;
+      if ((warp & 3) == 0 && lane == 0) AVSA_STAMP(1 + w, t, 3);
       // p = exp2(s * c - m) on pairs: one packed FMA, two EX2, one packed add, one bf16x2 convert per pair
       const uint64_t c2 = pack_f32x2(p.scale_log2, p.scale_log2);
       const uint64_t nm2 = pack_f32x2(-m_run, -m_run);
@@ -315,14 +379,21 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__
           pk[j] = pack_bf16x2(p0, p1);
         }
         tmem_st16(TM_S[w] + lane_off + c * 16, pk);
+        if (c == BLK / 64 - 1) {          // first half of the keys is in tensor memory: let the MMA warp start on it
+          tmem_wait_st();
+          tc_fence_before();
+          mbar_arrive(BAR(P_FULL + 2 * w));
+        }
       }
       float sa, sb;
       unpack_f32x2(add_f32x2(add_f32x2(sum2[0], sum2[1]), add_f32x2(sum2[2], sum2[3])), sa, sb);
       const float sum = sa + sb;
       l_run += sum;
+      if ((warp & 3) == 0 && lane == 0) AVSA_STAMP(1 + w, t, 4);
       tmem_wait_st();
       tc_fence_before();
-      mbar_arrive(BAR(P_FULL + w));
+      mbar_arrive(BAR(P_FULL + 2 * w + 1));
+      if ((warp & 3) == 0 && lane == 0) AVSA_STAMP(1 + w, t, 5);
     }
     // publish this group's statistics, then merge the two halves of the key axis
     stats[(w * 2 + 0) * 128 + row] = m_run;

@@ -25,6 +25,14 @@ static int launch_sparse_attn(int B, int H, int N, const avsa_bf16_4d& q, const 
 
 using namespace avsa;
 
+#ifdef AVSA_TRACE
+// Debug builds only: device buffer that receives the pipeline time stamps of CTA (0,0,0).
+static long long* g_trace_buffer = nullptr;
+extern "C" __attribute__((visibility("default"))) void avsa_debug_set_trace(long long* device_buffer) {
+  g_trace_buffer = device_buffer;
+}
+#endif
+
 extern "C" size_t avsa_sparse_self_attn_workspace_bytes(int B, int H, int N, int d, int blk) {
   if (B <= 0 || H <= 0 || N <= 0 || d <= 0 || blk <= 0) return 0;
   return kStatusBytes;
@@ -53,6 +61,9 @@ extern "C" int avsa_sparse_self_attn(int B, int H, int N, int d, int blk, avsa_b
   prm.NQT = prm.NKB = (N + blk - 1) / blk;
   const float scale = softmax_scale != 0.f ? softmax_scale : 1.0f / sqrtf(static_cast<float>(d));
   prm.scale_log2 = scale * 1.4426950408889634f;
+#ifdef AVSA_TRACE
+  prm.trace = g_trace_buffer;
+#endif
   clear_status_kernel<<<1, 1, 0, st>>>(prm.status);
   if (d == 128) return launch_sparse_attn<128, 128>(B, H, N, q, k, v, o_bf16, prm, st);
   return launch_sparse_attn<64, 64>(B, H, N, q, k, v, o_bf16, prm, st);
