@@ -2,7 +2,8 @@
 // (Eq. 10) and the first pass of the cross-attention (Eq. 1).
 //
 // One CTA per work item = one query tile and a list of key tiles.  Warp roles:
-//   warp 0      TMA producer: Q tile once, then the listed K and V tiles through two 3-stage rings
+//   warp 0      TMA producer: Q tile once, then the listed K tiles through a 3-stage ring
+//   warp 3      TMA producer: the listed V tiles through a 3-stage ring
 //   warp 1      MMA issuer: S = Q K^T (operands in shared memory) and O += P V (P in tensor memory)
 //   warp 2      tensor-memory allocation
 //   warps 4-7   softmax group 0: even tiles of the list, accumulator O0
@@ -182,38 +183,36 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__
 
   // The four service warps (0-3) give registers to the eight softmax warps (4-11); each role
   // changes its own budget as the first thing it does.
-  if (warp == 0) {
-    // ------------------------------------------------------------------ TMA producer
+  if (warp == 0 || warp == 3) {
+    // ------------------------------------------------------------------ TMA producers: warp 0 K (and Q), warp 3 V
     asm volatile("setmaxnreg.dec.sync.aligned.u32 64;");
-    if (lane == 0) {
+    const bool is_k = (warp == 0);
+    const CUtensorMap* tm = is_k ? &tmk : &tmv;
+    const int FULL = is_k ? K_FULL : V_FULL, EMPTY = is_k ? K_EMPTY : V_EMPTY;
+    const uint32_t base = smem_u32(smem + (is_k ? L::kK : L::kV));
+    if (is_k && lane == 0) {
       mbar_expect_tx(BAR(Q_FULL), BLK * D * 2);
       for (int pn = 0; pn < NPANEL; pn++)
         tma_load_4d(smem_u32(smem + L::kQ) + pn * QPANEL_BYTES, &tmq, BAR(Q_FULL), pn * 64, qt * BLK, h, b);
     }
+    int s = 0, fpar = 0;     // stage, and the parity of the "empty" phase to wait for once the ring has wrapped
     for (int t0 = 0; t0 < cnt; t0 += 32) {
       int mine = kb0 + t0 + lane;
       if (MODE == MODE_LIST) mine = (t0 + lane < cnt) ? list[t0 + lane] : 0;
       const int nn = min(32, cnt - t0);
       for (int j = 0; j < nn; j++) {
         const int kb = __shfl_sync(0xffffffffu, mine, j);
+        const int t = t0 + j;
         if (lane == 0) {
-          const int t = t0 + j, s = t % kStages, f = t / kStages;
           bool ok = true;
-          if (f > 0) ok = wait_or_abort(K_EMPTY + s, (f - 1) & 1, kWhereKEmpty, t);
+          if (t >= kStages) ok = wait_or_abort(EMPTY + s, fpar, is_k ? kWhereKEmpty : kWhereVEmpty, t);
           if (ok) {
-            mbar_expect_tx(BAR(K_FULL + s), L::kTileBytes);
+            mbar_expect_tx(BAR(FULL + s), L::kTileBytes);
             for (int pn = 0; pn < NPANEL; pn++)
-              tma_load_4d(smem_u32(smem + L::kK) + s * L::kTileBytes + pn * PANEL_BYTES, &tmk, BAR(K_FULL + s), pn * 64,
-                          kb * BLK, h, b);
-          }
-          if (ok && f > 0) ok = wait_or_abort(V_EMPTY + s, (f - 1) & 1, kWhereVEmpty, t);
-          if (ok) {
-            mbar_expect_tx(BAR(V_FULL + s), L::kTileBytes);
-            for (int pn = 0; pn < NPANEL; pn++)
-              tma_load_4d(smem_u32(smem + L::kV) + s * L::kTileBytes + pn * PANEL_BYTES, &tmv, BAR(V_FULL + s), pn * 64,
-                          kb * BLK, h, b);
+              tma_load_4d(base + s * L::kTileBytes + pn * PANEL_BYTES, tm, BAR(FULL + s), pn * 64, kb * BLK, h, b);
           }
         }
+        if (++s == kStages) { s = 0; if (t >= kStages) fpar ^= 1; }
       }
       if (__any_sync(0xffffffffu, misc[1] != 0u)) break;
     }
@@ -240,12 +239,11 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__
       bool ok = wait_all(Q_FULL, 0, kWhereQFull, 0);
       int sk = 0, fk = 0;      // stage / fill parity of the tile whose S is issued
       int sv = 0, fv = 0;      // same for the tile whose P V is issued
+      if (ok) ok = wait_all(K_FULL + 0, 0, kWhereKFull, 0);
       for (int t = 0; t <= cnt && ok; t++) {
         if (t < cnt) {
+          // K tile t has been waited for already (end of the previous iteration): issue at once
           const int w = t & 1;
-          if (leader) AVSA_STAMP(0, t, 5);
-          ok = wait_all(K_FULL + sk, fk, kWhereKFull, t);
-          if (!ok) break;
           tc_fence_after();
           const uint32_t k_lo = k_lo0 + sk * (L::kTileBytes >> 4);
           const uint32_t tm_s = tmem_u + (w << 7);
@@ -264,22 +262,29 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__
           __syncwarp();
           if (++sk == kStages) { sk = 0; fk ^= 1; }
         }
+        // Waits whose data arrived long ago are taken here, in the shadow of the running softmax, so that
+        // nothing but the wait for P stands between P's arrival and the next two MMA batches.
+        if (t >= 1) {
+          ok = wait_all(V_FULL + sv, fv, kWhereVFull, t - 1);
+          if (!ok) break;
+        }
+        if (t + 1 < cnt) {
+          ok = wait_all(K_FULL + sk, fk, kWhereKFull, t + 1);
+          if (!ok) break;
+        }
         if (t >= 1) {
           const int u = t - 1, w = u & 1, i = u >> 1;
-          if (leader) AVSA_STAMP(0, u, 2);
           // P arrives in two halves of the key axis: the first half of the product starts while the
           // softmax group is still exponentiating the second half
+          if (leader) AVSA_STAMP(0, u, 2);
           ok = wait_all(P_FULL + 2 * w, i & 1, kWherePFull, u);
-          if (!ok) break;
-          if (leader) AVSA_STAMP(0, u, 3);
-          ok = wait_all(V_FULL + sv, fv, kWhereVFull, u);
           if (!ok) break;
           tc_fence_after();
           const uint32_t v_lo = v_lo0 + sv * (L::kTileBytes >> 4);
           const uint32_t tm_p = tmem_u + (w << 7), tm_o = tmem_u + 256u + (w << 7);
           const uint32_t acc0 = i > 0 ? 1u : 0u;
           if (leader) {
-            AVSA_STAMP(0, u, 6);
+            AVSA_STAMP(0, u, 3);
 #pragma unroll
             for (int ks = 0; ks < BLK / 32; ks++)
               umma_ts(tm_o, tm_p + ks * 8, desc64(v_lo + ks * (2048 >> 4)), idesc_pv, ks > 0 ? 1u : acc0);
@@ -302,7 +307,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__
       if (ok && leader) umma_commit(BAR(FINAL));
       __syncwarp();
     }
-  } else if (warp < 4) {
+  } else if (warp == 2) {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 64;");
   } else {
     // ------------------------------------------------------------------ softmax groups + epilogue
@@ -333,14 +338,16 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__
         for (int j = 0; j < BLK; j++)
           if (j >= ragged_valid) s[j] = 0xff800000u;
       }
-      float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // four independent chains
+      float mx8[8];                                                  // eight independent chains
 #pragma unroll
-      for (int j = 0; j < BLK; j += 8) {
+      for (int u = 0; u < 8; u++) mx8[u] = fmaxf(__uint_as_float(s[2 * u]), __uint_as_float(s[2 * u + 1]));
 #pragma unroll
-        for (int u = 0; u < 4; u++)
-          mx4[u] = max3f(mx4[u], __uint_as_float(s[j + 2 * u]), __uint_as_float(s[j + 2 * u + 1]));
+      for (int j = 16; j < BLK; j += 16) {
+#pragma unroll
+        for (int u = 0; u < 8; u++)
+          mx8[u] = max3f(mx8[u], __uint_as_float(s[j + 2 * u]), __uint_as_float(s[j + 2 * u + 1]));
       }
-      const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+      const float mx = fmaxf(max3f(mx8[0], mx8[1], mx8[2]), fmaxf(max3f(mx8[3], mx8[4], mx8[5]), fmaxf(mx8[6], mx8[7])));
       const float m_new = fmaxf(m_run, mx * p.scale_log2);
       const bool need = (m_new - m_run) > kRescaleThreshold;     // true on the first tile (m_run = -inf)
       float factor = 1.f;
