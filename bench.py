@@ -27,6 +27,7 @@ import torch
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
+from paper_2608_15522_b200 import dist_timing as dt  # noqa: E402
 from paper_2608_15522_b200 import workloads as wl  # noqa: E402
 
 METRIC = "dense-equiv TFLOP/s of protected sparse video attn (layer-step: cross-attn scores + mask + sparse attn)"
@@ -172,19 +173,13 @@ def run_reference(args, w):
 # ------------------------------------------------------------------------------------------------ our arm
 def run_ours(args, w):
     from paper_2608_15522_b200 import binding as av
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank, local_rank, world = dt.world()
     if not torch.cuda.is_available():
         raise RuntimeError("bench.py needs a CUDA device: the path has no CPU fallback")
     av.load_library()
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist_mod
-        dist = dist_mod
-        dist.init_process_group("nccl", device_id=dev)
+    dist = dt.init("nccl", dev)
 
     seed = rank      # every rank owns an independent layer (replica): weak scaling, no collective on the data path
     q, k, v = wl.make_self_qkv(w, seed, dev)
@@ -211,10 +206,7 @@ def run_ours(args, w):
         av.avsa_sparse_self_attn(q, k, v, m["col_idx"], m["col_cnt"], w.blk, o=o, ws=ws3)
 
     def barrier():
-        torch.cuda.synchronize()
-        if dist is not None:
-            dist.barrier()
-        torch.cuda.synchronize()
+        dt.barrier(dist, dev)
 
     for _ in range(max(args.warmup, 3)):
         step()
@@ -300,16 +292,13 @@ def run_ours(args, w):
     e2e_ms = a.elapsed_time(b) / e2e_steps
 
     # ---- max over ranks
-    times = torch.tensor([total_ms, e2e_ms], dtype=torch.float64, device=dev)
-    if dist is not None:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    total_ms, e2e_ms = float(times[0]), float(times[1])
+    total_ms, e2e_ms = dt.max_over_ranks(dist, [total_ms, e2e_ms], dev)
     ms_per_step = total_ms / args.steps
     if rank == 0:
         peaks, peak_kind = load_peaks()
         fl_dense = dense_flops(w)
         fl_exec = pairs * 4.0 * w.blk * w.blk * w.d
-        value = world * fl_dense / (ms_per_step * 1e-3) / 1e12
+        value = dt.whole_job_rate(fl_dense, world, ms_per_step) / 1e12
         achieved = fl_exec / (t_attn * 1e-3) / 1e12
         peak = float(peaks.get("bf16_tflops", FALLBACK_PEAKS["bf16_tflops"]))
         sustained = float(peaks.get("bf16_tflops_sustained", FALLBACK_PEAKS["bf16_tflops_sustained"]))
@@ -358,7 +347,7 @@ def run_ours(args, w):
                             "cross_attn_scores_frac": cross_bytes / (t_cross * 1e-3) / 1e9 / hbm,
                             "peak_gbs": hbm, "peak_source": peak_kind},
             "cpu_baseline": cpu,
-            "e2e": {"value": world * fl_dense / (e2e_ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
+            "e2e": {"value": dt.whole_job_rate(fl_dense, world, e2e_ms) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
                     "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
             "gpu_launches": KERNELS_PER_STEP * args.steps,
             "clocks": clocks,
@@ -369,6 +358,93 @@ def run_ours(args, w):
         dist.destroy_process_group()
 
 
+def time_layer_step(av, w, seed, dev, n_iter=3, token_exact=False):
+    """Per-call CUDA-event times (ms, median of n_iter) of one layer-step on freshly generated tensors."""
+    q, k, v = wl.make_self_qkv(w, seed, dev)
+    qa, kc, vc = wl.make_cross_qkv(w, seed, dev)
+    n_protect = av.avsa_count_from_percent(w.protect_pct, w.n_video)
+    k_keep = max(1, av.avsa_count_from_percent(w.keep_pct, w.n_blocks))
+    gamma = 1.0 / (w.H * w.n_audio)
+    flags = av.AVSA_PROTECT_TOKENS if token_exact else av.AVSA_PROTECT_ROWS
+    o_a, lse, s, ws1 = av.avsa_cross_attn_scores(qa, kc, vc, score_gamma=gamma)
+    m = av.avsa_build_block_mask(q, k, s, n_protect, k_keep, w.blk, flags=flags)
+    o, _, ws3 = av.avsa_sparse_self_attn(q, k, v, m["col_idx"], m["col_cnt"], w.blk)
+    ws4 = av.avsa_protected_rows_attn(q, k, v, m["prot_tok"], n_protect, w.blk, o) if token_exact else None
+    rows = []
+    for _ in range(n_iter):
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(5)]
+        ev[0].record()
+        av.avsa_cross_attn_scores(qa, kc, vc, scores=s, score_gamma=gamma, o=o_a, lse=lse, ws=ws1)
+        ev[1].record()
+        av.avsa_build_block_mask(q, k, s, n_protect, k_keep, w.blk, flags=flags, out=m, ws=m["ws"])
+        ev[2].record()
+        av.avsa_sparse_self_attn(q, k, v, m["col_idx"], m["col_cnt"], w.blk, o=o, ws=ws3)
+        ev[3].record()
+        if token_exact:
+            av.avsa_protected_rows_attn(q, k, v, m["prot_tok"], n_protect, w.blk, o, ws=ws4)
+        ev[4].record()
+        torch.cuda.synchronize()
+        rows.append([ev[i].elapsed_time(ev[i + 1]) for i in range(4)])
+    t = np.median(np.array(rows), axis=0)
+    t_dense = None
+    try:
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.nn.functional.scaled_dot_product_attention(q, k, v)
+        a.record()
+        torch.nn.functional.scaled_dot_product_attention(q, k, v)
+        b.record(); torch.cuda.synchronize()
+        t_dense = a.elapsed_time(b)
+    except Exception:
+        pass
+    NB = w.n_blocks
+    pairs = int(m["col_cnt"].sum().item())
+    executed = (pairs * w.blk * w.blk + (w.B * w.H * n_protect * float(w.n_video) if token_exact else 0.0)) / (
+        w.B * w.H * float(w.n_video) ** 2)
+    return {"cross_ms": float(t[0]), "mask_ms": float(t[1]), "sparse_ms": float(t[2]), "protected_rows_ms": float(t[3]),
+            "attn_ms": float(t[2] + t[3]), "dense_library_ms": t_dense, "executed_fraction": executed,
+            "protected_blocks": int(m["prot_blk"].sum().item()), "n_blocks": NB}
+
+
+def run_sweep(args, w):
+    """Keep ratio x protected fraction grid on one workload (the mid-length sweep of the benchmark plan)."""
+    from paper_2608_15522_b200 import binding as av
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    out = []
+    for keep in (10, 25, 50):
+        for prot in (0, 5, 20):
+            for token_exact in (False, True):
+                if token_exact and prot == 0:
+                    continue
+                r = time_layer_step(av, w.with_ratios(keep, prot), 0, dev, token_exact=token_exact)
+                r.update(keep_pct=keep, protect_pct=prot, protection="tokens" if token_exact else "blocks")
+                if r["dense_library_ms"]:
+                    r["attn_speedup_vs_dense"] = r["dense_library_ms"] / r["attn_ms"]
+                out.append(r)
+    print(json.dumps({"sweep": w.name, "rows": out}))
+
+
+def run_loop(args, w):
+    """Multi-step denoising loop: fresh seeded tensors per (step, layer), mask rebuilt every step from that step's
+    cross-attention scores; reports the summed attention time against dense and the per-kernel shares."""
+    from paper_2608_15522_b200 import binding as av
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    tot = {"cross_ms": 0.0, "mask_ms": 0.0, "sparse_ms": 0.0, "protected_rows_ms": 0.0, "dense_library_ms": 0.0}
+    n = 0
+    for step in range(args.loop_steps):
+        for layer in range(args.loop_layers):
+            r = time_layer_step(av, w, wl.loop_seed(step, layer), dev, n_iter=1, token_exact=args.token_exact)
+            for key in tot:
+                tot[key] += r[key] or 0.0
+            n += 1
+    ours = tot["cross_ms"] + tot["mask_ms"] + tot["sparse_ms"] + tot["protected_rows_ms"]
+    print(json.dumps({"loop": w.name, "steps": args.loop_steps, "layers": args.loop_layers, "layer_steps": n,
+                      "protection": "tokens" if args.token_exact else "blocks", "total_ms": tot, "ours_ms": ours,
+                      "speedup_vs_dense_library": tot["dense_library_ms"] / ours if ours else None,
+                      "share": {k: v / ours for k, v in tot.items() if k != "dense_library_ms"}}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -377,9 +453,23 @@ def main():
     ap.add_argument("--workload", default="ovi", choices=wl.all_workload_names())
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--keep-pct", type=int, default=None)
+    ap.add_argument("--protect-pct", type=int, default=None)
+    ap.add_argument("--sweep", action="store_true", help="keep x protect grid on the chosen workload (one JSON line)")
+    ap.add_argument("--loop", action="store_true", help="multi-step denoising loop on the chosen workload")
+    ap.add_argument("--loop-steps", type=int, default=8)
+    ap.add_argument("--loop-layers", type=int, default=30)
+    ap.add_argument("--token-exact", action="store_true", help="loop mode: token-exact protection instead of blocks")
     args = ap.parse_args()
     w = wl.WORKLOADS[args.workload]
-    if args.impl == "reference":
+    if args.keep_pct is not None or args.protect_pct is not None:
+        w = w.with_ratios(args.keep_pct if args.keep_pct is not None else w.keep_pct,
+                          args.protect_pct if args.protect_pct is not None else w.protect_pct)
+    if args.sweep:
+        run_sweep(args, w)
+    elif args.loop:
+        run_loop(args, w)
+    elif args.impl == "reference":
         run_reference(args, w)
     else:
         run_ours(args, w)
