@@ -73,78 +73,99 @@ __global__ void __launch_bounds__(256) pool_kernel(const __nv_bfloat16* __restri
 }
 
 // ------------------------------------------------------------------------------------------------
-// (ii) block scores Bs[bh, i, j] = qbar[bh,i,:] . kbar[bh,j,:] * scale.  64x64 tile per CTA; both
-// operand tiles are brought into shared memory in one shot (all loads in flight at once), stored
-// channel-major so that each thread reads its 4 rows / 4 columns as one float4; 128 threads x (8x4)
-// outputs, channels summed in ascending order.
+// (ii) block scores Bs[bh, i, j] = qbar[bh,i,:] . kbar[bh,j,:] * scale.  The pooled means are fp32 and the
+// scores feed a top-k, so the product keeps fp32 accuracy: every operand is split into two tf32 halves
+// (x = hi + lo exactly to 2^-22) and three tensor-core products a_lo*b_hi + a_hi*b_lo + a_hi*b_hi are
+// accumulated in fp32 (warp-level m16n8k8 MMAs; the problem is far too small for the tcgen05 path).
+// 64x64 tile per CTA, 4 warps x (32x32), both operand tiles staged row-major in shared memory.
 // ------------------------------------------------------------------------------------------------
-constexpr int kScorePitch = 64 + 4;
+__device__ __forceinline__ void split_tf32(float x, uint32_t& hi, uint32_t& lo) {
+  asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(hi) : "f"(x));
+  const float r = x - __uint_as_float(hi);
+  asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(lo) : "f"(r));
+}
+__device__ __forceinline__ void mma_tf32(float (&d)[4], const uint32_t (&a)[4], const uint32_t (&b)[2]) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]));
+}
+
 template <int D>
 __global__ void __launch_bounds__(128) block_score_kernel(const float* __restrict__ qbar,
                                                           const float* __restrict__ kbar, float* __restrict__ bs,
                                                           int NB, float scale) {
+  constexpr int PITCH = D + 4;     // floats; keeps 16-byte alignment and makes fragment loads conflict-free
   extern __shared__ __align__(16) float score_smem[];
-  float(*sq)[kScorePitch] = reinterpret_cast<float(*)[kScorePitch]>(score_smem);
-  float(*sk)[kScorePitch] = reinterpret_cast<float(*)[kScorePitch]>(score_smem + D * kScorePitch);
-  const int bh = blockIdx.z, i0 = blockIdx.y * 64, j0 = blockIdx.x * 64;
-  const float* qb = qbar + static_cast<int64_t>(bh) * NB * D;
-  const float* kb = kbar + static_cast<int64_t>(bh) * NB * D;
+  float* sq = score_smem;
+  float* sk = score_smem + 64 * PITCH;
   // Launched as an ordinary stream-ordered kernel: it starts only after both the token select and the
   // pooling kernel (which may overlap each other) have finished.  The list kernel behind it may be
   // scheduled early and waits for this grid.
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-#pragma unroll 1
-  for (int half = 0; half < 2; half++) {
-    const int r = threadIdx.x % 64, cg = threadIdx.x / 64 + 2 * half;
-    float4 vq[D / 16], vk[D / 16];
-#pragma unroll
-    for (int it = 0; it < D / 16; it++) {
-      const int c4 = cg + 4 * it;
-      vq[it] = (i0 + r < NB) ? __ldg(reinterpret_cast<const float4*>(qb + static_cast<int64_t>(i0 + r) * D) + c4)
-                             : make_float4(0.f, 0.f, 0.f, 0.f);
-      vk[it] = (j0 + r < NB) ? __ldg(reinterpret_cast<const float4*>(kb + static_cast<int64_t>(j0 + r) * D) + c4)
-                             : make_float4(0.f, 0.f, 0.f, 0.f);
-    }
-#pragma unroll
-    for (int it = 0; it < D / 16; it++) {
-      const int c = (cg + 4 * it) * 4;
-      sq[c][r] = vq[it].x; sq[c + 1][r] = vq[it].y; sq[c + 2][r] = vq[it].z; sq[c + 3][r] = vq[it].w;
-      sk[c][r] = vk[it].x; sk[c + 1][r] = vk[it].y; sk[c + 2][r] = vk[it].z; sk[c + 3][r] = vk[it].w;
-    }
+  const int bh = blockIdx.z, i0 = blockIdx.y * 64, j0 = blockIdx.x * 64;
+  const float* qb = qbar + static_cast<int64_t>(bh) * NB * D;
+  const float* kb = kbar + static_cast<int64_t>(bh) * NB * D;
+  for (int e = threadIdx.x; e < 64 * (D / 4); e += 128) {
+    const int r = e / (D / 4), c4 = e % (D / 4);
+    const float4 vq = (i0 + r < NB) ? __ldg(reinterpret_cast<const float4*>(qb + static_cast<int64_t>(i0 + r) * D) + c4)
+                                    : make_float4(0.f, 0.f, 0.f, 0.f);
+    const float4 vk = (j0 + r < NB) ? __ldg(reinterpret_cast<const float4*>(kb + static_cast<int64_t>(j0 + r) * D) + c4)
+                                    : make_float4(0.f, 0.f, 0.f, 0.f);
+    *reinterpret_cast<float4*>(sq + r * PITCH + c4 * 4) = vq;
+    *reinterpret_cast<float4*>(sk + r * PITCH + c4 * 4) = vk;
   }
   __syncthreads();
-  const int tx = threadIdx.x % 16, ty = threadIdx.x / 16;     // 16 x 8 threads, 8 rows x 4 columns each
-  float acc[8][4];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = lane >> 2, t = lane & 3;
+  const int wr = (warp >> 1) * 32, wc = (warp & 1) * 32;     // this warp's 32x32 corner inside the tile
+  float acc[2][4][4];
 #pragma unroll
-  for (int a = 0; a < 8; a++)
+  for (int mi = 0; mi < 2; mi++)
 #pragma unroll
-    for (int c = 0; c < 4; c++) acc[a][c] = 0.f;
-#pragma unroll 4
-  for (int c = 0; c < D; c++) {
-    const float4 a0 = *reinterpret_cast<const float4*>(&sq[c][ty * 8]);
-    const float4 a1 = *reinterpret_cast<const float4*>(&sq[c][ty * 8 + 4]);
-    const float4 bv = *reinterpret_cast<const float4*>(&sk[c][tx * 4]);
-    const float a[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
-    const float bq[4] = {bv.x, bv.y, bv.z, bv.w};
+    for (int ni = 0; ni < 4; ni++)
 #pragma unroll
-    for (int t = 0; t < 8; t++)
+      for (int r = 0; r < 4; r++) acc[mi][ni][r] = 0.f;
+#pragma unroll 2
+  for (int k0 = 0; k0 < D; k0 += 8) {
+    uint32_t ah[2][4], al[2][4], bhh[4][2], bl[4][2];
 #pragma unroll
-      for (int u = 0; u < 4; u++) acc[t][u] = fmaf(a[t], bq[u], acc[t][u]);
-  }
-#pragma unroll
-  for (int t = 0; t < 8; t++) {
-    const int i = i0 + ty * 8 + t;
-    if (i >= NB) continue;
-    float* dst = bs + (static_cast<int64_t>(bh) * NB + i) * NB + j0 + tx * 4;
-    if (j0 + tx * 4 + 3 < NB && (NB & 3) == 0) {
-      *reinterpret_cast<float4*>(dst) = make_float4(acc[t][0] * scale, acc[t][1] * scale, acc[t][2] * scale,
-                                                    acc[t][3] * scale);
-    } else {
-#pragma unroll
-      for (int u = 0; u < 4; u++)
-        if (j0 + tx * 4 + u < NB) dst[u] = acc[t][u] * scale;
+    for (int mi = 0; mi < 2; mi++) {
+      const float* base = sq + (wr + mi * 16 + g) * PITCH + k0 + t;
+      split_tf32(base[0], ah[mi][0], al[mi][0]);
+      split_tf32(base[8 * PITCH], ah[mi][1], al[mi][1]);
+      split_tf32(base[4], ah[mi][2], al[mi][2]);
+      split_tf32(base[8 * PITCH + 4], ah[mi][3], al[mi][3]);
     }
+#pragma unroll
+    for (int ni = 0; ni < 4; ni++) {
+      const float* base = sk + (wc + ni * 8 + g) * PITCH + k0 + t;
+      split_tf32(base[0], bhh[ni][0], bl[ni][0]);
+      split_tf32(base[4], bhh[ni][1], bl[ni][1]);
+    }
+#pragma unroll
+    for (int mi = 0; mi < 2; mi++)
+#pragma unroll
+      for (int ni = 0; ni < 4; ni++) {
+        mma_tf32(acc[mi][ni], al[mi], bhh[ni]);     // small terms first
+        mma_tf32(acc[mi][ni], ah[mi], bl[ni]);
+        mma_tf32(acc[mi][ni], ah[mi], bhh[ni]);
+      }
   }
+#pragma unroll
+  for (int mi = 0; mi < 2; mi++)
+#pragma unroll
+    for (int half = 0; half < 2; half++) {
+      const int i = i0 + wr + mi * 16 + g + half * 8;
+      if (i >= NB) continue;
+#pragma unroll
+      for (int ni = 0; ni < 4; ni++) {
+        const int j = j0 + wc + ni * 8 + 2 * t;
+        float* dst = bs + (static_cast<int64_t>(bh) * NB + i) * NB + j;
+        if (j < NB) dst[0] = acc[mi][ni][half * 2] * scale;
+        if (j + 1 < NB) dst[1] = acc[mi][ni][half * 2 + 1] * scale;
+      }
+    }
 }
 
 // Adds one warp's digits to a shared-memory histogram.  When every participating lane holds the same
@@ -466,7 +487,7 @@ extern "C" int avsa_build_block_mask(int B, int H, int N, int d, int blk, avsa_b
     cfg.numAttrs = 1;
     const int64_t qsb = q.stride_b, qsh = q.stride_h, qsn = q.stride_n, ksb = k.stride_b, ksh = k.stride_h,
                   ksn = k.stride_n;
-    const size_t score_smem = static_cast<size_t>(2) * d * kScorePitch * sizeof(float);
+    const size_t score_smem = static_cast<size_t>(2) * 64 * (d + 4) * sizeof(float);
     cudaError_t e;
     if (d == 128) {
       e = cudaLaunchKernelEx(&cfg, pool_kernel<128>, qp, qsb, qsh, qsn, kp, ksb, ksh, ksn, qbar, kbar, H, N, blk);

@@ -103,3 +103,71 @@ def test_ovi_mask_full_and_sparse_attention_sampled_blocks(ovi):
             want_o, want_l = orc.masked_attention_rows(_np64(q[0, h, lo:hi]), kh, vh, cols, w.blk)
             _close(_np64(o[0, h, lo:hi]), want_o, f"O head {h} block {i}")
             _close(_np64(lse[0, h, lo:hi]), want_l, f"lse head {h} block {i}")
+
+
+def _check_workload_sampled(w, seed, heads, n_blocks_each, token_exact=False):
+    """Whole path on a full-size workload; mask bit-exact everywhere, attention on sampled query blocks."""
+    dev = torch.device("cuda", 0)
+    q, k, v = wl.make_self_qkv(w, seed, dev)
+    qa, kc, vc = wl.make_cross_qkv(w, seed, dev)
+    NB = w.n_blocks
+    n_protect = av.avsa_count_from_percent(w.protect_pct, w.n_video)
+    k_keep = max(1, av.avsa_count_from_percent(w.keep_pct, NB))
+    _, _, s, ws1 = av.avsa_cross_attn_scores(qa, kc, vc, score_gamma=1.0 / (w.H * w.n_audio))
+    assert av.avsa_read_status(ws1)[0] == av.AVSA_OK
+    assert abs(float(s.sum()) - w.B) < 2e-3 * w.B
+    flags = av.AVSA_PROTECT_TOKENS if token_exact else av.AVSA_PROTECT_ROWS
+    m = av.avsa_build_block_mask(q, k, s, n_protect, k_keep, w.blk, flags=flags)
+    bs_gpu = m["block_scores"].cpu().numpy()
+    idx, cnt, ptok, pblk = orc.build_block_mask(bs_gpu, s.cpu().numpy(), n_protect, k_keep, w.blk, w.n_video,
+                                                protect_rows=not token_exact)
+    assert np.array_equal(m["prot_tok"].cpu().numpy(), ptok)
+    assert np.array_equal(m["prot_blk"].cpu().numpy(), pblk)
+    assert np.array_equal(m["col_cnt"].cpu().numpy(), cnt)
+    assert np.array_equal(m["col_idx"].cpu().numpy(), idx)
+    o, lse, ws = av.avsa_sparse_self_attn(q, k, v, m["col_idx"], m["col_cnt"], w.blk, want_lse=True)
+    assert av.avsa_read_status(ws)[0] == av.AVSA_OK
+    if token_exact:
+        ws2 = av.avsa_protected_rows_attn(q, k, v, m["prot_tok"], n_protect, w.blk, o, lse=lse)
+        assert av.avsa_read_status(ws2)[0] == av.AVSA_OK
+    rng = np.random.default_rng(seed)
+    prot = np.nonzero(pblk[0])[0]
+    unprot = np.nonzero(pblk[0] == 0)[0]
+    blocks = [0, NB - 1]
+    if len(prot):
+        blocks += rng.choice(prot, min(n_blocks_each, len(prot)), replace=False).tolist()
+    if len(unprot):
+        blocks += rng.choice(unprot, min(n_blocks_each, len(unprot)), replace=False).tolist()
+    for h in heads:
+        qh, kh, vh = _np64(q[0, h]), _np64(k[0, h]), _np64(v[0, h])
+        for i in blocks:
+            lo, hi = i * w.blk, min((i + 1) * w.blk, w.n_video)
+            cols = [int(c) for c in idx[0, h, i, : cnt[0, h, i]]]
+            want_o, want_l = orc.masked_attention_rows(qh[lo:hi], kh, vh, cols, w.blk)
+            if token_exact:                                   # Eq. 11: protected rows are dense rows
+                rows = np.nonzero(ptok[0, lo:hi])[0]
+                if len(rows):
+                    d_o, d_l = orc.masked_attention_rows(qh[lo:hi][rows], kh, vh, list(range(NB)), w.blk)
+                    want_o[rows], want_l[rows] = d_o, d_l
+            _close(_np64(o[0, h, lo:hi]), want_o, f"{w.name} O head {h} block {i}")
+            _close(_np64(lse[0, h, lo:hi]), want_l, f"{w.name} lse head {h} block {i}")
+    return pblk, cnt
+
+
+@pytest.mark.parametrize("keep,protect", [(10, 0), (25, 5), (50, 20)])
+def test_mid_sweep_points(keep, protect):
+    w = wl.WORKLOADS["mid"].with_ratios(keep, protect)
+    pblk, cnt = _check_workload_sampled(w, 1, heads=(0, 17), n_blocks_each=2)
+    assert (w.n_video, w.n_blocks) == (17856, 140)
+    if protect == 0:
+        assert pblk.sum() == 0 and (cnt == av.avsa_count_from_percent(keep, 140)).all()
+
+
+def test_mid_token_exact_protection():
+    _check_workload_sampled(wl.WORKLOADS["mid"].with_ratios(25, 5), 2, heads=(5,), n_blocks_each=2, token_exact=True)
+
+
+def test_ltx_class_long_sequence():
+    w = wl.WORKLOADS["ltx"]
+    assert (w.n_video, w.n_blocks, w.n_audio) == (49152, 384, 512)
+    _check_workload_sampled(w, 0, heads=(0, 31), n_blocks_each=2)
