@@ -106,15 +106,21 @@ __global__ void __launch_bounds__(128) block_score_kernel(const float* __restric
   const int bh = blockIdx.z, i0 = blockIdx.y * 64, j0 = blockIdx.x * 64;
   const float* qb = qbar + static_cast<int64_t>(bh) * NB * D;
   const float* kb = kbar + static_cast<int64_t>(bh) * NB * D;
-  for (int e = threadIdx.x; e < 64 * (D / 4); e += 128) {
+  // both 64 x D tiles go straight from global to shared memory, every 16-byte piece in flight at once
+  // (rows beyond NB are zero-filled by a zero source size)
+#pragma unroll
+  for (int it = 0; it < 64 * (D / 4) / 128; it++) {
+    const int e = it * 128 + threadIdx.x;
     const int r = e / (D / 4), c4 = e % (D / 4);
-    const float4 vq = (i0 + r < NB) ? __ldg(reinterpret_cast<const float4*>(qb + static_cast<int64_t>(i0 + r) * D) + c4)
-                                    : make_float4(0.f, 0.f, 0.f, 0.f);
-    const float4 vk = (j0 + r < NB) ? __ldg(reinterpret_cast<const float4*>(kb + static_cast<int64_t>(j0 + r) * D) + c4)
-                                    : make_float4(0.f, 0.f, 0.f, 0.f);
-    *reinterpret_cast<float4*>(sq + r * PITCH + c4 * 4) = vq;
-    *reinterpret_cast<float4*>(sk + r * PITCH + c4 * 4) = vk;
+    const bool qv = (i0 + r < NB), kv = (j0 + r < NB);
+    const float* gq = qb + static_cast<int64_t>(qv ? i0 + r : 0) * D + c4 * 4;
+    const float* gk = kb + static_cast<int64_t>(kv ? j0 + r : 0) * D + c4 * 4;
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(static_cast<uint32_t>(
+                     __cvta_generic_to_shared(sq + r * PITCH + c4 * 4))), "l"(gq), "r"(qv ? 16 : 0) : "memory");
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(static_cast<uint32_t>(
+                     __cvta_generic_to_shared(sk + r * PITCH + c4 * 4))), "l"(gk), "r"(kv ? 16 : 0) : "memory");
   }
+  asm volatile("cp.async.wait_all;" ::: "memory");
   __syncthreads();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 2, t = lane & 3;
@@ -364,15 +370,32 @@ __global__ void __launch_bounds__(128) row_select_kernel(const float* __restrict
     want = k_keep;
     for (int pass = 0; pass < 4; pass++) {
       const int shift = 24 - 8 * pass;
+      // digit range of the keys still in play: when they all share the digit (typical for the leading byte)
+      // the pass needs no histogram at all
+      uint32_t dmin = 255u, dmax = 0u;
+#pragma unroll
+      for (int j = 0; j < KPL; j++) {
+        const bool in = (j * 32 + lane < NB) && ((keys[j] & mask) == prefix);
+        const uint32_t dg = (keys[j] >> shift) & 255u;
+        if (in) {
+          dmin = min(dmin, dg);
+          dmax = max(dmax, dg);
+        }
+      }
+      dmin = __reduce_min_sync(0xffffffffu, dmin);
+      dmax = __reduce_max_sync(0xffffffffu, dmax);
+      if (dmin == dmax) {
+        prefix |= dmin << shift;
+        mask |= 255u << shift;
+        continue;
+      }
 #pragma unroll
       for (int i = 0; i < 8; i++) bins[i * 32 + lane] = 0;
       __syncwarp();
 #pragma unroll
       for (int j = 0; j < KPL; j++) {
-        if (j * 32 < NB) {
-          const bool in = (j * 32 + lane < NB) && ((keys[j] & mask) == prefix);
-          warp_hist_add(bins, in, (keys[j] >> shift) & 255u, lane);
-        }
+        const bool in = (j * 32 + lane < NB) && ((keys[j] & mask) == prefix);
+        if (in) atomicAdd(&bins[(keys[j] >> shift) & 255u], 1);
       }
       __syncwarp();
       int dg, ab, ib;
