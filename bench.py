@@ -267,6 +267,13 @@ def run_ours(args, w):
     except Exception:
         t_dense_lib = None
     t_token_exact = time_fn(token_exact_attn, 5)
+    # ---- cache-reuse indicators (Eq. 12-15) on feature maps of the layer's size ([B, N, H*d] views of Q/K buffers)
+    C = w.H * w.d
+    yv, yhv = q.view(w.B, w.n_video, C), k.view(w.B, w.n_video, C)
+    ya, yha = qa.view(w.B, w.n_audio, C), qa.view(w.B, w.n_audio, C)
+    ind_out, ws_ind = av.avsa_cache_indicators(yv, yhv, ya, yha, m["prot_tok"], s, s)
+    t_ind = time_fn(lambda: av.avsa_cache_indicators(yv, yhv, ya, yha, m["prot_tok"], s, s, out=ind_out, ws=ws_ind), 10)
+    ind_bytes = 2.0 * w.B * (w.n_video + w.n_audio) * C * 2
     del idx_all, cnt_all
 
     # ---- end to end through the public API with host buffers (pinned), copies inside the timed region
@@ -336,6 +343,10 @@ def run_ours(args, w):
                 "kappa_plus_rho": (w.keep_pct + w.protect_pct) / 100.0,
                 "speedup_vs_dense": dense_best / t_token_exact,
                 "dense_equiv_tflops": fl_dense / (t_token_exact * 1e-3) / 1e12},
+            "cache_indicators": {"ms": t_ind, "gbs": ind_bytes / (t_ind * 1e-3) / 1e9,
+                                 "frac_of_hbm_peak": ind_bytes / (t_ind * 1e-3) / 1e9 / hbm,
+                                 "note": "Eq. 12-15 on [B,N,H*d] feature maps; reads both maps once; L2 not flushed "
+                                         "between repetitions but the 406 MB exceed it"},
             "executed_tflops": achieved,
             "roofline": {"kernel": "attn_fwd_kernel<128,128,MODE_LIST> (avsa_sparse_self_attn)", "bound": "tensor",
                          "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,

@@ -144,6 +144,26 @@ AVSA_API int avsa_protected_rows_attn(int B, int H, int N, int d, int blk, avsa_
 AVSA_API size_t avsa_protected_rows_attn_workspace_bytes(int B, int H, int N, int d, int blk, int n_protect);
 
 /*
+ * (5) Cache-reuse indicators -- Eq. 12 (stream-wise feature change), Eq. 13 (change over the protected video
+ * tokens), Eq. 14 (saliency drift) and Eq. 15 (their maximum against the threshold).
+ *
+ *   y_v, yhat_v  bf16 [B,Nv,C] contiguous: current and cached block outputs of the video stream
+ *   y_a, yhat_a  bf16 [B,Na,C] contiguous: the same for the audio stream
+ *   prot_tok     uint8 [B,Nv] protected-token flags (NULL: no protected set, dp = 0)
+ *   s_cur, s_anchor  fp32 [B,Nv] current and anchor saliency maps (both NULL: ds = 0)
+ *   out          fp32 [B,8]: dv, da, dp, ds, dsync = max(dv, da, lambda_p*dp, lambda_s*ds), reuse (1.0 iff
+ *                dsync < tau), two unused slots
+ *   dv = sum|y - yhat| / (sum|y| + eps), likewise da and dp; ds = 1 - <s,s^>/(|s||s^| + eps).
+ * C must be a multiple of 8.  Sums are taken in a fixed order (bit-reproducible).  The paper's settings are
+ * lambda_p = 0.5, lambda_s = 0.1, tau = 0.2.
+ */
+AVSA_API int avsa_cache_indicators(int B, int Nv, int Na, int C, const void* y_v, const void* yhat_v, const void* y_a,
+                                   const void* yhat_a, const uint8_t* prot_tok, const float* s_cur,
+                                   const float* s_anchor, float lambda_p, float lambda_s, float tau, float eps,
+                                   float* out, void* ws, size_t ws_bytes, void* stream);
+AVSA_API size_t avsa_cache_indicators_workspace_bytes(int B, int Nv, int Na, int C);
+
+/*
  * Allocation-free variant of avsa_build_block_mask.  The paper has no counterpart; this is a
  * convenience of the library for callers that have no device allocator to draw a workspace from:
  * code that runs after its host application has frozen its memory budget, extensions loaded into

@@ -15,6 +15,7 @@ What follows the paper and what is this build's reading of it:
   per-head top-k) is this build's choice.  PARITY UNPINNED against the paper's own system for this
   rule; the functions are pinned against brute force and closed forms only.
 * ``protected_attention_token_exact``               -- Eq. 9 / Eq. 11 on tokens (dense rows for protected tokens).
+* ``cache_indicators``                             -- Eq. 12-15 (relative L1 changes, saliency drift, their maximum).
 * ``protected_blocks``, ``build_block_mask``       -- Eq. 9 lifted from tokens to blocks: a block is
   protected iff it holds at least one protected token (a superset of the token-level rule).
 
@@ -251,3 +252,30 @@ def dense_attention(q, k, v, scale=None):
     """Eq. 5: softmax(q k^T * scale) v for [B,H,N,d] tensors."""
     o, lse, _ = cross_attention(q, k, v, scale)
     return o, lse
+
+
+# ------------------------------------------------------------------------------------------------
+# Eq. 12-15: synchronization-aware cache-reuse indicators
+# ------------------------------------------------------------------------------------------------
+def cache_indicators(y_v, yhat_v, y_a, yhat_a, prot_tok=None, s_cur=None, s_anchor=None, lambda_p=0.5, lambda_s=0.1,
+                     tau=0.2, eps=1e-6):
+    """One batch item.  y_v, yhat_v [Nv,C]; y_a, yhat_a [Na,C]; prot_tok [Nv] flags; s_cur, s_anchor [Nv].
+
+    Returns dict(dv, da, dp, ds, dsync, reuse):  Eq. 12 relative L1 change of each stream, Eq. 13 the same over
+    the protected video rows, Eq. 14 one minus the cosine of the saliency maps, Eq. 15 their weighted maximum
+    and the reuse decision dsync < tau.
+    """
+    y_v = np.asarray(y_v, np.float64); yhat_v = np.asarray(yhat_v, np.float64)
+    y_a = np.asarray(y_a, np.float64); yhat_a = np.asarray(yhat_a, np.float64)
+    dv = np.abs(y_v - yhat_v).sum() / (np.abs(y_v).sum() + eps)
+    da = np.abs(y_a - yhat_a).sum() / (np.abs(y_a).sum() + eps)
+    dp = 0.0
+    if prot_tok is not None:
+        rows = np.nonzero(np.asarray(prot_tok))[0]
+        dp = np.abs(y_v[rows] - yhat_v[rows]).sum() / (np.abs(y_v[rows]).sum() + eps)
+    ds = 0.0
+    if s_cur is not None and s_anchor is not None:
+        a = np.asarray(s_cur, np.float64); c = np.asarray(s_anchor, np.float64)
+        ds = 1.0 - float(a @ c) / (np.sqrt(float(a @ a)) * np.sqrt(float(c @ c)) + eps)
+    dsync = max(dv, da, lambda_p * dp, lambda_s * ds)
+    return dict(dv=dv, da=da, dp=dp, ds=ds, dsync=dsync, reuse=bool(dsync < tau))

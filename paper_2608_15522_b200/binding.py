@@ -33,6 +33,7 @@ EXPORTS = (
     "avsa_build_block_mask", "avsa_build_block_mask_workspace_bytes", "avsa_build_block_mask_static",
     "avsa_sparse_self_attn", "avsa_sparse_self_attn_workspace_bytes",
     "avsa_protected_rows_attn", "avsa_protected_rows_attn_workspace_bytes",
+    "avsa_cache_indicators", "avsa_cache_indicators_workspace_bytes",
     "avsa_count_from_percent", "avsa_read_status", "avsa_status_string", "avsa_version",
 )
 
@@ -80,6 +81,10 @@ def load_library() -> ctypes.CDLL:
     lib.avsa_protected_rows_attn.restype = i
     lib.avsa_protected_rows_attn_workspace_bytes.argtypes = [i, i, i, i, i, i]
     lib.avsa_protected_rows_attn_workspace_bytes.restype = sz
+    lib.avsa_cache_indicators.argtypes = [i, i, i, i, vp, vp, vp, vp, vp, vp, vp, f, f, f, f, vp, vp, sz, vp]
+    lib.avsa_cache_indicators.restype = i
+    lib.avsa_cache_indicators_workspace_bytes.argtypes = [i, i, i, i]
+    lib.avsa_cache_indicators_workspace_bytes.restype = sz
     lib.avsa_count_from_percent.argtypes = [i, i]
     lib.avsa_count_from_percent.restype = i
     lib.avsa_read_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_int)]
@@ -276,3 +281,28 @@ def avsa_protected_rows_attn(q, k, v, prot_tok, n_protect, blk, o, lse=None, sof
                                       _ptr(lse), float(softmax_scale), _ptr(ws), ws.numel(), _stream(dev))
     _check(st, "avsa_protected_rows_attn")
     return ws
+
+
+def avsa_cache_indicators_workspace_bytes(B, Nv, Na, C) -> int:
+    return int(load_library().avsa_cache_indicators_workspace_bytes(B, Nv, Na, C))
+
+
+def avsa_cache_indicators(y_v, yhat_v, y_a, yhat_a, prot_tok=None, s_cur=None, s_anchor=None, lambda_p=0.5,
+                          lambda_s=0.1, tau=0.2, eps=1e-6, out=None, ws=None):
+    """Eq. 12-15.  y_v/yhat_v bf16 [B,Nv,C], y_a/yhat_a bf16 [B,Na,C] (contiguous).  Returns (out [B,8], ws) with
+    out[:, :6] = dv, da, dp, ds, dsync, reuse."""
+    lib = load_library()
+    B, Nv, C = y_v.shape
+    Na = y_a.shape[1]
+    dev = y_v.device
+    for t in (y_v, yhat_v, y_a, yhat_a):
+        if t.dtype != torch.bfloat16 or not t.is_contiguous() or not t.is_cuda:
+            raise ValueError("expected contiguous CUDA bf16 tensors")
+    if out is None:
+        out = torch.empty((B, 8), dtype=torch.float32, device=dev)
+    ws = _workspace(avsa_cache_indicators_workspace_bytes(B, Nv, Na, C), dev, ws)
+    st = lib.avsa_cache_indicators(B, Nv, Na, C, _ptr(y_v), _ptr(yhat_v), _ptr(y_a), _ptr(yhat_a), _ptr(prot_tok),
+                                   _ptr(s_cur), _ptr(s_anchor), float(lambda_p), float(lambda_s), float(tau),
+                                   float(eps), _ptr(out), _ptr(ws), ws.numel(), _stream(dev))
+    _check(st, "avsa_cache_indicators")
+    return out, ws

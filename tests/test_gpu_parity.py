@@ -342,6 +342,38 @@ def test_token_exact_protection_matches_oracle(name):
     assert torch.equal(before, o)
 
 
+# ------------------------------------------------------------------------------------------- Eq. 12-15
+@pytest.mark.parametrize("Nv,Na,C", [(390, 40, 384), (2070, 72, 512), (5, 3, 8)])
+def test_cache_indicators_match_oracle(Nv, Na, C):
+    B = 2
+    g = torch.Generator().manual_seed(Nv)
+    y_v = torch.randn((B, Nv, C), generator=g).bfloat16()
+    yhat_v = (y_v.float() + 0.2 * torch.randn((B, Nv, C), generator=g)).bfloat16()
+    y_a = torch.randn((B, Na, C), generator=g).bfloat16()
+    yhat_a = (y_a.float() + 0.05 * torch.randn((B, Na, C), generator=g)).bfloat16()
+    prot = (torch.rand((B, Nv), generator=g) < 0.1).to(torch.uint8)
+    prot[:, 0] = 1
+    s_cur = torch.rand((B, Nv), generator=g)
+    s_anchor = (s_cur + 0.3 * torch.rand((B, Nv), generator=g)).float()
+    out, ws = av.avsa_cache_indicators(y_v.cuda(), yhat_v.cuda(), y_a.cuda(), yhat_a.cuda(), prot.cuda(), s_cur.cuda(),
+                                       s_anchor.cuda())
+    _status_ok(ws)
+    got = out.cpu().numpy()
+    for b in range(B):
+        want = orc.cache_indicators(_np64(y_v[b]), _np64(yhat_v[b]), _np64(y_a[b]), _np64(yhat_a[b]), prot[b].numpy(),
+                                    _np64(s_cur[b]), _np64(s_anchor[b]))
+        for i, key in enumerate(("dv", "da", "dp", "ds", "dsync")):
+            assert abs(got[b, i] - want[key]) <= 1e-4 * max(1.0, abs(want[key])), (b, key, got[b, i], want[key])
+        assert bool(got[b, 5]) == want["reuse"]
+    # no protected set and no saliency maps: those terms drop out
+    out2, _ = av.avsa_cache_indicators(y_v.cuda(), y_v.cuda(), y_a.cuda(), y_a.cuda())
+    assert np.allclose(out2.cpu().numpy()[:, :5], 0.0) and (out2.cpu().numpy()[:, 5] == 1.0).all()
+    # reproducible bit for bit
+    out3, _ = av.avsa_cache_indicators(y_v.cuda(), yhat_v.cuda(), y_a.cuda(), yhat_a.cuda(), prot.cuda(), s_cur.cuda(),
+                                       s_anchor.cuda())
+    assert torch.equal(out, out3)
+
+
 def test_host_side_argument_errors():
     w = wl.WORKLOADS["tiny"]
     q, k, v = (t.cuda() for t in wl.make_self_qkv(w, 0))

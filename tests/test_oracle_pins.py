@@ -355,3 +355,34 @@ def test_token_exact_protection_is_eq9_on_tokens():
         np.testing.assert_allclose(lse[0, h, prot], dense_lse[0, h, prot], rtol=1e-12)
         np.testing.assert_allclose(O[0, h, ~prot], sparse[0, h, ~prot], rtol=1e-12, atol=1e-13)   # Eq. 11, second case
     assert ptok.sum() == n_protect
+
+
+# ------------------------------------------------------------------------------- Eq. 12-15
+def test_cache_indicators_golden_and_closed_forms():
+    g = {}
+    with open(os.path.join(os.path.dirname(GOLDEN), "cache_indicators_example.txt")) as f:
+        for line in f:
+            if not line.startswith("#") and line.strip():
+                k, v = line.split()
+                g[k] = float(v)
+    r = orc.cache_indicators([[1, -2], [3, 4]], [[1, 0], [0, 4]], [[2, 2]], [[1, 3]], prot_tok=[0, 1],
+                             s_cur=[1, 0], s_anchor=[1, 1], eps=0.0)
+    for k in ("dv", "da", "dp", "ds", "dsync"):
+        assert abs(r[k] - g[k]) < 1e-15, k
+    assert r["reuse"] == bool(g["reuse"])
+    # identical features and parallel saliency maps: nothing changed, reuse
+    y = _rand((7, 4), 41); a = _rand((3, 4), 42); s = np.abs(_rand((7,), 43))
+    r = orc.cache_indicators(y, y, a, a, prot_tok=[1, 0, 0, 1, 0, 0, 0], s_cur=s, s_anchor=3.0 * s, eps=0.0)
+    assert r["dv"] == 0 and r["da"] == 0 and r["dp"] == 0 and abs(r["ds"]) < 1e-15 and r["reuse"]
+    # cache of zeros: relative change 1; orthogonal saliency maps: drift 1; scale invariance of the ratios
+    r = orc.cache_indicators(y, 0 * y, a, 0 * a, prot_tok=[0, 1, 0, 0, 0, 0, 0], s_cur=[1, 0, 0, 0, 0, 0, 0],
+                             s_anchor=[0, 1, 0, 0, 0, 0, 0], eps=0.0)
+    assert abs(r["dv"] - 1) < 1e-15 and abs(r["da"] - 1) < 1e-15 and abs(r["dp"] - 1) < 1e-15 and abs(r["ds"] - 1) < 1e-15
+    yh = y + 0.1 * _rand((7, 4), 44)
+    r1 = orc.cache_indicators(y, yh, a, a, eps=0.0)
+    r2 = orc.cache_indicators(5 * y, 5 * yh, a, a, eps=0.0)
+    assert abs(r1["dv"] - r2["dv"]) < 1e-15
+    # Eq. 15 is a weighted maximum: each term can be the binding one
+    assert orc.cache_indicators(y, yh, a, a + 10, eps=0.0)["dsync"] == orc.cache_indicators(y, yh, a, a + 10, eps=0.0)["da"]
+    r = orc.cache_indicators(y, y, a, a, s_cur=[1, 0, 0, 0, 0, 0, 0], s_anchor=[0, 1, 0, 0, 0, 0, 0], lambda_s=0.1, eps=0.0)
+    assert abs(r["dsync"] - 0.1) < 1e-15 and r["reuse"]            # 0.1 * 1 < tau = 0.2
