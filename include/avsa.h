@@ -77,7 +77,8 @@ typedef struct {
  * accumulates layers; score_beta = alpha with score_gamma = (1-alpha)/(H*Nq) is Eq. 4.
  * With score_beta == 0 the previous contents of scores are ignored (may be uninitialised).
  * o, lse and scores may each be NULL to skip that output (scores == NULL skips the second pass).
- * softmax_scale == 0 means 1/sqrt(d).  Nq <= 512.  The head sum is taken in a fixed order, so
+ * softmax_scale == 0 means 1/sqrt(d).  Nq <= 512 when scores are requested (any Nq otherwise, which serves the
+ * reverse, video->audio direction of the bidirectional pair).  The head sum is taken in a fixed order, so
  * results reproduce bit for bit.  `o` has strides (o_stride_b, o_stride_h, o_stride_n) = q's.
  */
 AVSA_API int avsa_cross_attn_scores(int B, int H, int Nq, int Nk, int d, avsa_bf16_4d q, avsa_bf16_4d k, avsa_bf16_4d v,

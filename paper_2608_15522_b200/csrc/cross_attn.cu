@@ -336,7 +336,8 @@ extern "C" int avsa_cross_attn_scores(int B, int H, int Nq, int Nk, int d, avsa_
                                       void* stream) {
   if (B <= 0 || H <= 0 || Nq <= 0 || Nk <= 0) return AVSA_ERR_INVALID_ARG;
   if (d != 64 && d != 128) return AVSA_ERR_UNSUPPORTED;
-  if (Nq > 512 || H > 65535 || B > 65535) return AVSA_ERR_UNSUPPORTED;
+  if (H > 65535 || B > 65535) return AVSA_ERR_UNSUPPORTED;
+  if (scores != nullptr && Nq > 512) return AVSA_ERR_UNSUPPORTED;   // the score pass keeps a head's queries on chip
   if (!tensor_ok(q, B, H) || !tensor_ok(k, B, H) || !tensor_ok(v, B, H)) return AVSA_ERR_INVALID_ARG;
   if (o_bf16 != nullptr && !aligned16(o_bf16)) return AVSA_ERR_INVALID_ARG;
   if (softmax_scale < 0.f || softmax_scale != softmax_scale) return AVSA_ERR_INVALID_ARG;

@@ -278,6 +278,24 @@ def test_cross_attention_long_query_axis_two_chunks():
     assert np.linalg.norm(_np64(s) - want_s) / np.linalg.norm(want_s) <= REL_L2
 
 
+@pytest.mark.parametrize("name", ["tiny", "medium128"])
+def test_cross_attention_reverse_direction_outputs(name):
+    """Video queries attending to audio keys (the other half of the bidirectional pair): outputs and LSE."""
+    w = wl.WORKLOADS[name]
+    qa, kc, vc = wl.make_cross_qkv(w, 3)
+    q_video, k_audio, v_audio = kc, qa, wl.make_cross_qkv(w, 4)[0]          # roles swapped; fresh audio values
+    want_o, want_lse, _ = orc.cross_attention(_np64(q_video), _np64(k_audio), _np64(v_audio))
+    o, lse, s, ws = av.avsa_cross_attn_scores(q_video.cuda(), k_audio.cuda(), v_audio.cuda(), want_scores=False)
+    _status_ok(ws)
+    assert s is None
+    _close(_np64(o), want_o, f"{name} reverse O")
+    _close(_np64(lse), want_lse, f"{name} reverse lse")
+    if w.n_video > 512:
+        with pytest.raises(av.AvsaError) as e:                               # scores need the queries on chip
+            av.avsa_cross_attn_scores(q_video.cuda(), k_audio.cuda(), v_audio.cuda())
+        assert e.value.status == av.AVSA_ERR_UNSUPPORTED
+
+
 # ------------------------------------------------------------------------------------------- whole path
 def test_whole_path_tiny_matches_oracle():
     w = wl.WORKLOADS["tiny"]
