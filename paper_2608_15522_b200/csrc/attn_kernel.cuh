@@ -16,6 +16,7 @@
 //             and TMA-stored; optional natural-log LSE.
 // MODE_RANGE  key tiles are a contiguous range (one split of the key axis); the output is a partial
 //             result (fp32 rows normalised by their own sum, plus the log2-domain LSE of the split).
+// MODE_RANGE_DIRECT  the whole key axis as one range (few keys): output written like MODE_LIST.
 #pragma once
 #include "avsa_common.cuh"
 #include "sm100_ptx.cuh"
@@ -26,7 +27,7 @@ constexpr int kAttnThreads = 384;
 constexpr int kStages = 3;
 constexpr float kRescaleThreshold = 8.0f;   // log2 units: O is rescaled only when a row max grew by more
 
-enum { MODE_LIST = 0, MODE_RANGE = 1 };
+enum { MODE_LIST = 0, MODE_RANGE = 1, MODE_RANGE_DIRECT = 2 };
 
 enum AttnWhere {
   kWhereQFull = 1, kWhereKEmpty, kWhereVEmpty, kWhereKFull, kWhereVFull, kWherePFull, kWhereSFull, kWhereFinal,
@@ -83,6 +84,8 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__
                 const __grid_constant__ CUtensorMap tmv, const __grid_constant__ CUtensorMap tmo,
                 const AttnParams p) {
   using L = AttnSmem<BLK, D>;
+  constexpr bool kListIn = (MODE == MODE_LIST);          // explicit list of key tiles (else a contiguous range)
+  constexpr bool kDirectOut = (MODE != MODE_RANGE);      // final bf16 tile + LSE (else a partial result)
   constexpr int NPANEL = D / 64;
   constexpr int PANEL_BYTES = BLK * 128;        // one 64-channel panel of a K/V tile
   constexpr int QPANEL_BYTES = 128 * 128;
@@ -92,7 +95,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__
   const int h = blockIdx.y, b = blockIdx.z;
   int qt, split = 0, kb0 = 0, cnt;
   const int32_t* list = nullptr;
-  if (MODE == MODE_LIST) {
+  if (kListIn) {
     qt = blockIdx.x;
     const int row_id = (b * p.H + h) * p.NQT + qt;
     list = p.col_idx + static_cast<int64_t>(row_id) * p.NKB;
@@ -103,12 +106,12 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__
     kb0 = split * p.tiles_per_split;
     cnt = min(p.NKB, kb0 + p.tiles_per_split) - kb0;
   }
-  const int item = ((b * p.H + h) * p.NQT + qt) * (MODE == MODE_LIST ? 1 : p.n_split) + split;
+  const int item = ((b * p.H + h) * p.NQT + qt) * (kListIn ? 1 : p.n_split) + split;
 
   // ---- validation: nothing is loaded through a bad list entry
   {
     int bad = (cnt < 1 || cnt > p.NKB) ? 1 : 0;
-    if (MODE == MODE_LIST) {
+    if (kListIn) {
       const int n = min(max(cnt, 0), p.NKB);
       for (int t = tid; t < n; t += kAttnThreads) {
         const int kb = list[t];
@@ -154,7 +157,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__
     prefetch_tmap(&tmq);
     prefetch_tmap(&tmk);
     prefetch_tmap(&tmv);
-    if (MODE == MODE_LIST) prefetch_tmap(&tmo);
+    if (kDirectOut) prefetch_tmap(&tmo);
   }
   if (warp == 2) {
     tmem_alloc(smem_u32(smem + L::kMisc), 512);
@@ -198,7 +201,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__
     int s = 0, fpar = 0;     // stage, and the parity of the "empty" phase to wait for once the ring has wrapped
     for (int t0 = 0; t0 < cnt; t0 += 32) {
       int mine = kb0 + t0 + lane;
-      if (MODE == MODE_LIST) mine = (t0 + lane < cnt) ? list[t0 + lane] : 0;
+      if (kListIn) mine = (t0 + lane < cnt) ? list[t0 + lane] : 0;
       const int nn = min(32, cnt - t0);
       for (int j = 0; j < nn; j++) {
         const int kb = __shfl_sync(0xffffffffu, mine, j);
@@ -316,7 +319,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__
     const int row = ((warp & 3) << 5) + lane;    // row of the tile == TMEM lane
     const uint32_t lane_off = static_cast<uint32_t>((warp & 3) * 32) << 16;
     const int nw = n_tiles[w];
-    const int last_kb = (MODE == MODE_LIST) ? list[cnt - 1] : kb0 + cnt - 1;
+    const int last_kb = (kListIn) ? list[cnt - 1] : kb0 + cnt - 1;
     const int ragged_valid = (last_kb == p.NKB - 1) ? (p.Nk - last_kb * BLK) : BLK;   // valid keys of the last tile
     float m_run = -INFINITY, l_run = 0.f;
     bool ok = true;
@@ -434,7 +437,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__
           if (have1) v[j] = fmaf(__uint_as_float(o1[j]), f1, v[j]);
         }
         if (row < BLK) {
-          if (MODE == MODE_LIST) {
+          if (kDirectOut) {
 #pragma unroll
             for (int g = 0; g < 4; g++) {
               const int col = col0 + g * 8;
@@ -455,18 +458,18 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__
       }
       if (w == 0 && row < BLK) {
         const float lse2 = m + log2f(Lsum);
-        if (MODE == MODE_LIST) {
+        if (kDirectOut) {
           if (p.lse != nullptr && qt * BLK + row < p.Nq)
             p.lse[(static_cast<int64_t>(b) * p.H + h) * p.Nq + qt * BLK + row] = lse2 * 0.6931471805599453f;
         } else {
           p.part_lse2[static_cast<int64_t>(item) * BLK + row] = lse2;
         }
       }
-      if (MODE == MODE_LIST) fence_proxy_async();
+      if (kDirectOut) fence_proxy_async();
     }
     tc_fence_before();
     asm volatile("bar.sync 1, 256;" ::: "memory");
-    if (MODE == MODE_LIST && ok && warp == 4 && lane == 0) {
+    if (kDirectOut && ok && warp == 4 && lane == 0) {
       for (int pn = 0; pn < NPANEL; pn++)
         tma_store_4d(&tmo, smem_u32(smem + L::kQ) + pn * QPANEL_BYTES, pn * 64, qt * BLK, h, b);
       tma_store_commit();

@@ -200,6 +200,201 @@ colsum_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ C
   if (warp == 2) tmem_dealloc(tmem, 512);
 }
 
+// ------------------------------------------------------------------------------------------------
+// pass 2, many queries / few keys (the reverse, video->audio direction): the key tiles of one (batch, head)
+// stay in shared memory (at most 4 x 128 keys) and the queries stream through a 3-stage ring in chunks of
+// 128 together with their slice of log2-domain LSEs.  Units (query chunk, key tile) alternate between two
+// tensor-memory buffers and two groups of 128 threads (one thread per key row), each thread accumulating
+// the column sum of its key over the CTA's range of query chunks.
+//   partial[(range*2 + group)][b,h,key]; the head-sum kernel adds ranges, groups and heads in a fixed order.
+// ------------------------------------------------------------------------------------------------
+constexpr int kRevStages = 3;
+constexpr int kRevLseSlots = 5;      // LSE slices outlive their query stage by up to two units of exponentials
+
+struct ColsumRevParams {
+  const float* lse2;       // [B,H,NQC*128] log2-domain LSE, +inf beyond Nq
+  float* partial;          // [n_range*2][B,H,Nk]
+  StatusRecord* status;
+  int H, Nk, NKT, NQC;     // key tiles (<= 4) and query chunks of 128
+  int n_range, chunks_per_range;
+  float scale_log2;
+};
+
+template <int D>
+struct ColsumRevSmem {
+  static constexpr int kTile = 128 * D * 2;
+  static constexpr int kQ = 0;                              // ring of query chunks
+  __host__ __device__ static int k_offset() { return kRevStages * kTile; }      // NKT resident key tiles follow
+  __host__ __device__ static int lse_offset(int NKT) { return k_offset() + NKT * kTile; }
+  __host__ __device__ static int bars_offset(int NKT) { return lse_offset(NKT) + kRevLseSlots * 512; }
+  static constexpr int kNumBars = 1 + 2 * kRevStages + 4;
+  static int total(int NKT) { return bars_offset(NKT) + 128 + 16; }
+};
+
+enum ColRevWhere { kRevKFull = 51, kRevQEmpty, kRevQFull, kRevSEmpty, kRevSFull };
+
+template <int D>
+__global__ void __launch_bounds__(kColThreads, 1)
+colsum_rev_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUtensorMap tmk,
+                  const ColsumRevParams p) {
+  using L = ColsumRevSmem<D>;
+  constexpr int NPANEL = D / 64;
+  constexpr int PANEL_BYTES = 128 * 128;
+  extern __shared__ __align__(1024) uint8_t smem[];
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int range = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+  const int c_begin = range * p.chunks_per_range;
+  const int nchunk = min(p.NQC, c_begin + p.chunks_per_range) - c_begin;
+  const int item = (b * p.H + h) * p.n_range + range;
+  const int NKT = p.NKT;
+  if (nchunk <= 0) return;
+  if ((smem_u32(smem) & 1023u) != 0u) {
+    if (tid == 0) report_status(p.status, AVSA_ERR_CUDA, kWhereSmemAlign, item, 0);
+    return;
+  }
+  const int bars_off = L::bars_offset(NKT);
+  const uint32_t bar0 = smem_u32(smem + bars_off);
+  auto BAR = [&](int i) { return bar0 + static_cast<uint32_t>(i) * 8u; };
+  constexpr int K_FULL = 0, Q_FULL = 1, Q_EMPTY = 1 + kRevStages, S_FULL = 1 + 2 * kRevStages, S_EMPTY = S_FULL + 2;
+  const float* lse_slots = reinterpret_cast<const float*>(smem + L::lse_offset(NKT));
+  volatile uint32_t* misc = reinterpret_cast<volatile uint32_t*>(smem + bars_off + 128);
+  const float* lse2_bh = p.lse2 + (static_cast<int64_t>(b) * p.H + h) * (static_cast<int64_t>(p.NQC) * 128);
+
+  if (tid == 0) {
+    mbar_init(BAR(K_FULL), 1);
+    for (int s = 0; s < kRevStages; s++) {
+      mbar_init(BAR(Q_FULL + s), 1);
+      mbar_init(BAR(Q_EMPTY + s), 1);
+    }
+    for (int g = 0; g < 2; g++) {
+      mbar_init(BAR(S_FULL + g), 1);
+      mbar_init(BAR(S_EMPTY + g), 128);
+    }
+    misc[1] = 0u;
+    fence_mbar_init();
+    prefetch_tmap(&tmq);
+    prefetch_tmap(&tmk);
+  }
+  if (warp == 2) {
+    tmem_alloc(smem_u32(const_cast<uint32_t*>(misc)), 256);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = misc[0];
+
+  auto wait_or_abort = [&](int bar, uint32_t parity, int where, int aux) -> bool {
+    if (mbar_try_wait(BAR(bar), parity)) return true;
+    if (misc[1] != 0u) return false;
+    if (mbar_wait(BAR(bar), parity)) return true;
+    report_status(p.status, AVSA_ERR_TIMEOUT, where, item, aux);
+    misc[1] = 1u;
+    return false;
+  };
+
+  const int n_units = nchunk * NKT;
+  if (warp == 0) {
+    if (lane == 0) {
+      mbar_expect_tx(BAR(K_FULL), NKT * L::kTile);
+      for (int kt = 0; kt < NKT; kt++)
+        for (int pn = 0; pn < NPANEL; pn++)
+          tma_load_4d(smem_u32(smem) + L::k_offset() + kt * L::kTile + pn * PANEL_BYTES, &tmk, BAR(K_FULL), pn * 64,
+                      kt * 128, h, b);
+      bool ok = true;
+      for (int c = 0; c < nchunk && ok; c++) {
+        const int s = c % kRevStages, f = c / kRevStages;
+        if (f > 0) ok = wait_or_abort(Q_EMPTY + s, (f - 1) & 1, kRevQEmpty, c);
+        if (!ok) break;
+        mbar_expect_tx(BAR(Q_FULL + s), L::kTile + 512);
+        for (int pn = 0; pn < NPANEL; pn++)
+          tma_load_4d(smem_u32(smem) + L::kQ + s * L::kTile + pn * PANEL_BYTES, &tmq, BAR(Q_FULL + s), pn * 64,
+                      (c_begin + c) * 128, h, b);
+        bulk_load_1d(smem_u32(smem) + L::lse_offset(NKT) + (c % kRevLseSlots) * 512,
+                     lse2_bh + static_cast<int64_t>(c_begin + c) * 128, 512, BAR(Q_FULL + s));
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      const uint32_t idesc = make_idesc_bf16(128, 128, 0, 0);
+      bool ok = wait_or_abort(K_FULL, 0, kRevKFull, 0);
+      for (int c = 0; c < nchunk && ok; c++) {
+        const int s = c % kRevStages, f = c / kRevStages;
+        ok = wait_or_abort(Q_FULL + s, f & 1, kRevQFull, c);
+        if (!ok) break;
+        const uint32_t q_addr = smem_u32(smem) + L::kQ + s * L::kTile;
+        for (int kt = 0; kt < NKT && ok; kt++) {
+          const int u = c * NKT + kt, g = u & 1, i = u >> 1;
+          if (i > 0) ok = wait_or_abort(S_EMPTY + g, (i - 1) & 1, kRevSEmpty, u);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t k_addr = smem_u32(smem) + L::k_offset() + kt * L::kTile;
+#pragma unroll
+          for (int ks = 0; ks < D / 16; ks++) {
+            const uint64_t ad = make_sdesc(k_addr + (ks >> 2) * PANEL_BYTES + (ks & 3) * 32, 16, 1024);
+            const uint64_t bd = make_sdesc(q_addr + (ks >> 2) * PANEL_BYTES + (ks & 3) * 32, 16, 1024);
+            umma_ss(tmem + g * 128, ad, bd, idesc, ks > 0 ? 1u : 0u);
+          }
+          umma_commit(BAR(S_FULL + g));
+        }
+        if (ok) umma_commit(BAR(Q_EMPTY + s));
+      }
+    }
+  } else if (warp >= 4) {
+    const int g = (warp - 4) >> 2;
+    const int row = ((warp & 3) << 5) + lane;
+    const uint32_t lane_off = static_cast<uint32_t>((warp & 3) * 32) << 16;
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+    bool ok = true;
+    for (int u = g; u < n_units && ok; u += 2) {
+      const int i = u >> 1, c = u / NKT, kt = u % NKT;
+      ok = wait_or_abort(S_FULL + g, i & 1, kRevSFull, u);
+      if (!ok) break;
+      tc_fence_after();
+      const float* l2 = lse_slots + (c % kRevLseSlots) * 128;
+      float sum0 = 0.f, sum1 = 0.f;
+      const uint32_t base = tmem + g * 128 + lane_off;
+#pragma unroll
+      for (int cc = 0; cc < 128; cc += 32) {
+        uint32_t s[32];
+        tmem_ld32(base + cc, s);
+        tmem_wait_ld();
+#pragma unroll
+        for (int j = 0; j < 32; j += 4) {
+          const float4 lv = *reinterpret_cast<const float4*>(l2 + cc + j);
+          sum0 += fast_exp2(fmaf(__uint_as_float(s[j]), p.scale_log2, -lv.x));
+          sum1 += fast_exp2(fmaf(__uint_as_float(s[j + 1]), p.scale_log2, -lv.y));
+          sum0 += fast_exp2(fmaf(__uint_as_float(s[j + 2]), p.scale_log2, -lv.z));
+          sum1 += fast_exp2(fmaf(__uint_as_float(s[j + 3]), p.scale_log2, -lv.w));
+        }
+      }
+      tc_fence_before();
+      mbar_arrive(BAR(S_EMPTY + g));
+      const float tot = sum0 + sum1;
+      if (kt == 0) acc[0] += tot; else if (kt == 1) acc[1] += tot; else if (kt == 2) acc[2] += tot; else acc[3] += tot;
+    }
+    const int64_t slot = static_cast<int64_t>(range) * 2 + g;
+    float* dst = p.partial + (slot * gridDim.z * p.H + static_cast<int64_t>(b) * p.H + h) * p.Nk;
+#pragma unroll
+    for (int kt = 0; kt < 4; kt++) {
+      const int key = kt * 128 + row;
+      if (kt < NKT && key < p.Nk) dst[key] = acc[kt];
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 2) tmem_dealloc(tmem, 256);
+}
+
+// lse2[bh][i] = lse[bh][i] * log2(e) for i < Nq, +inf up to the padded length (multiple of 128)
+__global__ void __launch_bounds__(256) lse_to_log2_kernel(const float* __restrict__ lse, int Nq, int Nq_pad, int BH,
+                                                          float* __restrict__ lse2) {
+  const int64_t idx = static_cast<int64_t>(blockIdx.x) * 256 + threadIdx.x;
+  if (idx >= static_cast<int64_t>(BH) * Nq_pad) return;
+  const int bh = static_cast<int>(idx / Nq_pad), i = static_cast<int>(idx % Nq_pad);
+  lse2[idx] = i < Nq ? lse[static_cast<int64_t>(bh) * Nq + i] * 1.4426950408889634f : INFINITY;
+}
+
 // scores[b,i] = beta * scores[b,i] + gamma * sum_h sum_ch partial[ch][b,h,i], heads in ascending order
 __global__ void __launch_bounds__(256) head_sum_kernel(const float* __restrict__ partial, int NCH, int B, int H,
                                                        int Nk, float beta, float gamma, float* __restrict__ scores) {
@@ -218,7 +413,9 @@ __global__ void __launch_bounds__(256) head_sum_kernel(const float* __restrict__
 struct CrossPlan {
   int blk, NQT, NKB, n_split, tps;           // pass 1 (key tiles of blk)
   int NKT, NCH, W, n_range, tpr;             // pass 2 (key tiles of 128)
-  size_t off_part_o, off_part_lse, off_lse, off_partial, total;
+  bool reverse;                              // pass 2 with the keys resident (Nq > 512, Nk <= 512)
+  int NQC, rev_ranges, rev_cpr, rev_slots;   // query chunks of 128, CTAs per (b,h), chunks per CTA, partial slots
+  size_t off_part_o, off_part_lse, off_lse, off_lse2, off_partial, total;
 };
 
 static CrossPlan make_cross_plan(int B, int H, int Nq, int Nk, int d) {
@@ -240,12 +437,22 @@ static CrossPlan make_cross_plan(int B, int H, int Nq, int Nk, int d) {
   if (want_range > c.NKT) want_range = c.NKT;
   c.tpr = (c.NKT + want_range - 1) / want_range;
   c.n_range = (c.NKT + c.tpr - 1) / c.tpr;
+  c.reverse = Nq > 512;
+  c.NQC = (Nq + 127) / 128;
+  int want_rev = target / (B * H);
+  if (want_rev < 1) want_rev = 1;
+  if (want_rev > c.NQC) want_rev = c.NQC;
+  c.rev_cpr = (c.NQC + want_rev - 1) / want_rev;
+  c.rev_ranges = (c.NQC + c.rev_cpr - 1) / c.rev_cpr;
+  c.rev_slots = c.rev_ranges * 2;
   size_t off = kStatusBytes;
   const size_t items = static_cast<size_t>(B) * H * c.NQT * c.n_split;
   c.off_part_o = off; off += align_up(items * c.blk * d * sizeof(float), 256);
   c.off_part_lse = off; off += align_up(items * c.blk * sizeof(float), 256);
   c.off_lse = off; off += align_up(static_cast<size_t>(B) * H * Nq * sizeof(float), 256);
-  c.off_partial = off; off += align_up(static_cast<size_t>(c.NCH) * B * H * Nk * sizeof(float), 256);
+  c.off_lse2 = off; off += c.reverse ? align_up(static_cast<size_t>(B) * H * c.NQC * 128 * sizeof(float), 256) : 0;
+  const size_t slots = c.reverse ? static_cast<size_t>(c.rev_slots) : static_cast<size_t>(c.NCH);
+  c.off_partial = off; off += align_up(slots * B * H * Nk * sizeof(float), 256);
   c.total = off;
   return c;
 }
@@ -283,15 +490,54 @@ static int run_cross(int B, int H, int Nq, int Nk, const avsa_bf16_4d& q, const 
     prm.NKB = c.NKB;
     prm.scale_log2 = scale * 1.4426950408889634f;
     dim3 grid(c.NQT * c.n_split, H, B);
-    attn_fwd_kernel<BLK, D, MODE_RANGE><<<grid, kAttnThreads, L::kTotal, st>>>(tq, tk, tv, tq, prm);
-    const int total_rows = B * H * Nq;
-    constexpr int RPB = 128 / (D / 4);
-    merge_splits_kernel<BLK, D><<<(total_rows + RPB - 1) / RPB, 128, 0, st>>>(
-        part_o, part_lse, c.n_split, c.NQT, Nq, H, total_rows, static_cast<__nv_bfloat16*>(o), q.stride_b, q.stride_h,
-        q.stride_n, lse, nullptr, 0, Nq);
+    if (c.n_split == 1 && o != nullptr) {
+      // the whole key axis fits one work item (few keys): write O and the LSE directly, no partials to merge
+      CUtensorMap to;
+      if (!encode_bf16_tile_map(&to, o, B, H, Nq, D, q.stride_b, q.stride_h, q.stride_n, BLK)) return AVSA_ERR_CUDA;
+      if (cudaFuncSetAttribute(attn_fwd_kernel<BLK, D, MODE_RANGE_DIRECT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               L::kTotal) != cudaSuccess)
+        return AVSA_ERR_CUDA;
+      prm.lse = lse;
+      attn_fwd_kernel<BLK, D, MODE_RANGE_DIRECT><<<grid, kAttnThreads, L::kTotal, st>>>(tq, tk, tv, to, prm);
+    } else {
+      attn_fwd_kernel<BLK, D, MODE_RANGE><<<grid, kAttnThreads, L::kTotal, st>>>(tq, tk, tv, tq, prm);
+      const int total_rows = B * H * Nq;
+      constexpr int RPB = 128 / (D / 4);
+      merge_splits_kernel<BLK, D><<<(total_rows + RPB - 1) / RPB, 128, 0, st>>>(
+          part_o, part_lse, c.n_split, c.NQT, Nq, H, total_rows, static_cast<__nv_bfloat16*>(o), q.stride_b, q.stride_h,
+          q.stride_n, lse, nullptr, 0, Nq);
+    }
   }
-  // ---- pass 2
-  if (scores != nullptr) {
+  // ---- pass 2, keys resident (many queries, at most 512 keys)
+  if (scores != nullptr && c.reverse) {
+    using L = ColsumRevSmem<D>;
+    float* lse2 = reinterpret_cast<float*>(ws + c.off_lse2);
+    const int64_t n2 = static_cast<int64_t>(B) * H * c.NQC * 128;
+    lse_to_log2_kernel<<<static_cast<unsigned>((n2 + 255) / 256), 256, 0, st>>>(lse, Nq, c.NQC * 128, B * H, lse2);
+    CUtensorMap tq, tk;
+    if (!encode_bf16_tile_map(&tq, q.ptr, B, H, Nq, D, q.stride_b, q.stride_h, q.stride_n, 128)) return AVSA_ERR_CUDA;
+    if (!encode_bf16_tile_map(&tk, k.ptr, B, H, Nk, D, k.stride_b, k.stride_h, k.stride_n, 128)) return AVSA_ERR_CUDA;
+    const int smem = L::total(c.NKT);
+    if (cudaFuncSetAttribute(colsum_rev_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess)
+      return AVSA_ERR_CUDA;
+    ColsumRevParams rp;
+    rp.lse2 = lse2;
+    rp.partial = partial;
+    rp.status = status;
+    rp.H = H;
+    rp.Nk = Nk;
+    rp.NKT = c.NKT;
+    rp.NQC = c.NQC;
+    rp.n_range = c.rev_ranges;
+    rp.chunks_per_range = c.rev_cpr;
+    rp.scale_log2 = scale * 1.4426950408889634f;
+    colsum_rev_kernel<D><<<dim3(c.rev_ranges, H, B), kColThreads, smem, st>>>(tq, tk, rp);
+    const int64_t n = static_cast<int64_t>(B) * Nk;
+    head_sum_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, st>>>(partial, c.rev_slots, B, H, Nk, beta, gamma,
+                                                                           scores);
+  }
+  // ---- pass 2, queries resident (at most 512 queries)
+  if (scores != nullptr && !c.reverse) {
     using L = ColsumSmem<D>;
     CUtensorMap tq, tk;
     if (!encode_bf16_tile_map(&tq, q.ptr, B, H, Nq, D, q.stride_b, q.stride_h, q.stride_n, c.W)) return AVSA_ERR_CUDA;
@@ -337,7 +583,8 @@ extern "C" int avsa_cross_attn_scores(int B, int H, int Nq, int Nk, int d, avsa_
   if (B <= 0 || H <= 0 || Nq <= 0 || Nk <= 0) return AVSA_ERR_INVALID_ARG;
   if (d != 64 && d != 128) return AVSA_ERR_UNSUPPORTED;
   if (H > 65535 || B > 65535) return AVSA_ERR_UNSUPPORTED;
-  if (scores != nullptr && Nq > 512) return AVSA_ERR_UNSUPPORTED;   // the score pass keeps a head's queries on chip
+  // the score pass keeps either the queries or the keys of a head on chip
+  if (scores != nullptr && Nq > 512 && Nk > 512) return AVSA_ERR_UNSUPPORTED;
   if (!tensor_ok(q, B, H) || !tensor_ok(k, B, H) || !tensor_ok(v, B, H)) return AVSA_ERR_INVALID_ARG;
   if (o_bf16 != nullptr && !aligned16(o_bf16)) return AVSA_ERR_INVALID_ARG;
   if (softmax_scale < 0.f || softmax_scale != softmax_scale) return AVSA_ERR_INVALID_ARG;

@@ -63,6 +63,27 @@ def test_ovi_cross_attention_sampled_heads(ovi):
     assert region[top].mean() > 0.9
 
 
+def test_ovi_reverse_direction_audio_saliency(ovi):
+    """Video queries, audio keys at full size: audio-token saliency (column sums over 32760 video queries)."""
+    w, _, (qa, kc, vc) = ovi
+    q_video, k_audio, v_audio = kc, qa, qa
+    gamma = 1.0 / (w.H * w.n_video)
+    o, lse, s, ws = av.avsa_cross_attn_scores(q_video, k_audio, v_audio, score_gamma=gamma)
+    assert av.avsa_read_status(ws)[0] == av.AVSA_OK
+    want_s = np.zeros((w.B, w.n_audio))
+    for h in range(w.H):
+        want_o, want_lse, A = orc.cross_attention(_np64(q_video[:, h:h + 1]), _np64(k_audio[:, h:h + 1]),
+                                                  _np64(v_audio[:, h:h + 1]))
+        want_s = orc.column_scores(A, s_prev=want_s, beta=1.0, gamma=gamma)
+        if h in (0, 23):
+            _close(_np64(o[:, h:h + 1]), want_o, f"reverse O head {h}")
+            _close(_np64(lse[:, h:h + 1]), want_lse, f"reverse lse head {h}")
+    got_s = _np64(s)
+    assert abs(got_s.sum() - 1.0) < 2e-3
+    assert np.linalg.norm(got_s - want_s) / np.linalg.norm(want_s) <= REL_L2
+    assert np.abs(got_s - want_s).max() <= MAX_ABS
+
+
 def test_ovi_mask_full_and_sparse_attention_sampled_blocks(ovi):
     w, (q, k, v), (qa, kc, vc) = ovi
     NB = w.n_blocks

@@ -278,22 +278,37 @@ def test_cross_attention_long_query_axis_two_chunks():
     assert np.linalg.norm(_np64(s) - want_s) / np.linalg.norm(want_s) <= REL_L2
 
 
-@pytest.mark.parametrize("name", ["tiny", "medium128"])
-def test_cross_attention_reverse_direction_outputs(name):
-    """Video queries attending to audio keys (the other half of the bidirectional pair): outputs and LSE."""
+@pytest.mark.parametrize("name", ["tiny", "small128", "medium128"])
+def test_cross_attention_reverse_direction(name):
+    """Video queries attending to audio keys (the other half of the bidirectional pair): outputs, LSE, and the
+    audio-token saliency as column sums over the video queries (handled "analogously", Sec. 4.1)."""
     w = wl.WORKLOADS[name]
     qa, kc, vc = wl.make_cross_qkv(w, 3)
     q_video, k_audio, v_audio = kc, qa, wl.make_cross_qkv(w, 4)[0]          # roles swapped; fresh audio values
-    want_o, want_lse, _ = orc.cross_attention(_np64(q_video), _np64(k_audio), _np64(v_audio))
-    o, lse, s, ws = av.avsa_cross_attn_scores(q_video.cuda(), k_audio.cuda(), v_audio.cuda(), want_scores=False)
+    want_o, want_lse, A = orc.cross_attention(_np64(q_video), _np64(k_audio), _np64(v_audio))
+    gamma = 1.0 / (w.H * w.n_video)
+    want_s = orc.column_scores(A, gamma=gamma)
+    o, lse, s, ws = av.avsa_cross_attn_scores(q_video.cuda(), k_audio.cuda(), v_audio.cuda(), score_gamma=gamma)
     _status_ok(ws)
-    assert s is None
     _close(_np64(o), want_o, f"{name} reverse O")
     _close(_np64(lse), want_lse, f"{name} reverse lse")
-    if w.n_video > 512:
-        with pytest.raises(av.AvsaError) as e:                               # scores need the queries on chip
-            av.avsa_cross_attn_scores(q_video.cuda(), k_audio.cuda(), v_audio.cuda())
-        assert e.value.status == av.AVSA_ERR_UNSUPPORTED
+    got_s = _np64(s)
+    assert got_s.shape == (w.B, w.n_audio)
+    assert abs(got_s.sum() - w.B) < 2e-3 * w.B
+    assert np.linalg.norm(got_s - want_s) / np.linalg.norm(want_s) <= REL_L2
+    assert np.abs(got_s - want_s).max() <= MAX_ABS
+    _, _, s2, _ = av.avsa_cross_attn_scores(q_video.cuda(), k_audio.cuda(), v_audio.cuda(), score_gamma=gamma)
+    assert torch.equal(s, s2)                                              # fixed summation order
+
+
+def test_cross_attention_scores_need_one_short_axis():
+    """Neither the queries nor the keys of a head fit on chip: the score pass is refused on the host."""
+    q = torch.zeros((1, 1, 1024, 128), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(av.AvsaError) as e:
+        av.avsa_cross_attn_scores(q, q, q)
+    assert e.value.status == av.AVSA_ERR_UNSUPPORTED
+    o, lse, s, ws = av.avsa_cross_attn_scores(q, q, q, want_scores=False)  # outputs alone are fine
+    _status_ok(ws)
 
 
 # ------------------------------------------------------------------------------------------- whole path
@@ -390,6 +405,24 @@ def test_cache_indicators_match_oracle(Nv, Na, C):
     out3, _ = av.avsa_cache_indicators(y_v.cuda(), yhat_v.cuda(), y_a.cuda(), yhat_a.cuda(), prot.cuda(), s_cur.cuda(),
                                        s_anchor.cuda())
     assert torch.equal(out, out3)
+
+
+def test_audio_branch_short_sequences():
+    """The audio branch (m = a in Eq. 8-10) is the same three calls on a short sequence: fewer tokens than one
+    block, and a two-block sequence with one protected block."""
+    for (H, d, blk, N, k_keep, n_protect) in ((2, 64, 64, 40, 1, 4), (3, 128, 128, 256, 1, 13)):
+        g = torch.Generator().manual_seed(N)
+        q, k, v = (torch.randn((1, H, N, d), generator=g).bfloat16() for _ in range(3))
+        s = torch.rand((1, N), generator=g)
+        m = av.avsa_build_block_mask(q.cuda(), k.cuda(), s.cuda(), n_protect, k_keep, blk)
+        idx, cnt, ptok, pblk = orc.build_block_mask(m["block_scores"].cpu().numpy(), s.numpy(), n_protect, k_keep, blk, N)
+        assert np.array_equal(m["col_idx"].cpu().numpy(), idx) and np.array_equal(m["col_cnt"].cpu().numpy(), cnt)
+        assert np.array_equal(m["prot_tok"].cpu().numpy(), ptok) and ptok.sum() == n_protect
+        o, lse, ws = av.avsa_sparse_self_attn(q.cuda(), k.cuda(), v.cuda(), m["col_idx"], m["col_cnt"], blk, want_lse=True)
+        _status_ok(ws)
+        want_o, want_l = orc.masked_attention(_np64(q), _np64(k), _np64(v), idx, cnt, blk)
+        _close(_np64(o), want_o, f"audio branch N={N} O")
+        _close(_np64(lse), want_l, f"audio branch N={N} lse")
 
 
 def test_host_side_argument_errors():
