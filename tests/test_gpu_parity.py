@@ -407,6 +407,46 @@ def test_cache_indicators_match_oracle(Nv, Na, C):
     assert torch.equal(out, out3)
 
 
+@pytest.mark.parametrize("B,H,N,d,blk", [(1, 1, 1, 128, 128), (2, 1, 129, 128, 128), (3, 2, 65, 64, 64), (1, 5, 640, 128, 128)])
+def test_degenerate_shapes_whole_path(B, H, N, d, blk):
+    """One token, a one-token tail block, several batch items, one head: every call against the oracle."""
+    g = torch.Generator().manual_seed(B * 1000 + N)
+    Na = 7
+    q, k, v = (torch.randn((B, H, N, d), generator=g).bfloat16() for _ in range(3))
+    qa = torch.randn((B, H, Na, d), generator=g).bfloat16()
+    NB = (N + blk - 1) // blk
+    n_protect, k_keep = min(N, 3), max(1, NB // 2)
+    gamma = 1.0 / (H * Na)
+    o_a, lse_a, s, ws = av.avsa_cross_attn_scores(qa.cuda(), k.cuda(), v.cuda(), score_gamma=gamma)
+    _status_ok(ws)
+    want_oa, want_la, A = orc.cross_attention(_np64(qa), _np64(k), _np64(v))
+    _close(_np64(o_a), want_oa, "cross O")
+    _close(_np64(lse_a), want_la, "cross lse")
+    want_s = orc.column_scores(A, gamma=gamma)
+    assert np.abs(_np64(s) - want_s).max() <= MAX_ABS and np.linalg.norm(_np64(s) - want_s) <= REL_L2 * np.linalg.norm(want_s)
+    m = av.avsa_build_block_mask(q.cuda(), k.cuda(), s, n_protect, k_keep, blk)
+    idx, cnt, ptok, pblk = orc.build_block_mask(m["block_scores"].cpu().numpy(), s.cpu().numpy(), n_protect, k_keep, blk, N)
+    want_bs = orc.block_scores(_np64(q), _np64(k), blk)
+    assert np.abs(m["block_scores"].cpu().numpy() - want_bs).max() <= 1e-4 * max(1.0, np.abs(want_bs).max())
+    assert np.array_equal(m["col_idx"].cpu().numpy(), idx) and np.array_equal(m["col_cnt"].cpu().numpy(), cnt)
+    assert np.array_equal(m["prot_tok"].cpu().numpy(), ptok) and np.array_equal(m["prot_blk"].cpu().numpy(), pblk)
+    o, lse, ws3 = av.avsa_sparse_self_attn(q.cuda(), k.cuda(), v.cuda(), m["col_idx"], m["col_cnt"], blk, want_lse=True)
+    _status_ok(ws3)
+    want_o, want_l = orc.masked_attention(_np64(q), _np64(k), _np64(v), idx, cnt, blk)
+    _close(_np64(o), want_o, "O")
+    _close(_np64(lse), want_l, "lse")
+    # token-exact variant on the same inputs
+    m2 = av.avsa_build_block_mask(q.cuda(), k.cuda(), s, n_protect, k_keep, blk, flags=av.AVSA_PROTECT_TOKENS)
+    o2, lse2, _ = av.avsa_sparse_self_attn(q.cuda(), k.cuda(), v.cuda(), m2["col_idx"], m2["col_cnt"], blk, want_lse=True)
+    ws4 = av.avsa_protected_rows_attn(q.cuda(), k.cuda(), v.cuda(), m2["prot_tok"], n_protect, blk, o2, lse=lse2)
+    _status_ok(ws4)
+    idx2, cnt2, ptok2, _ = orc.build_block_mask(m2["block_scores"].cpu().numpy(), s.cpu().numpy(), n_protect, k_keep, blk, N,
+                                                protect_rows=False)
+    want_o2, want_l2 = orc.protected_attention_token_exact(_np64(q), _np64(k), _np64(v), idx2, cnt2, ptok2, blk)
+    _close(_np64(o2), want_o2, "token-exact O")
+    _close(_np64(lse2), want_l2, "token-exact lse")
+
+
 def test_audio_branch_short_sequences():
     """The audio branch (m = a in Eq. 8-10) is the same three calls on a short sequence: fewer tokens than one
     block, and a two-block sequence with one protected block."""
