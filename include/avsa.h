@@ -51,6 +51,9 @@ typedef enum {
   AVSA_ERR_BAD_MASK = 6      /* device: a column list entry was out of range or not ascending */
 } avsa_status;
 
+/* Size of the status record area at the start of every workspace. */
+#define AVSA_STATUS_BYTES 256
+
 /* bf16 tensor [B,H,N,d], d contiguous; strides in elements. */
 typedef struct {
   const void* ptr;
@@ -120,6 +123,13 @@ AVSA_API size_t avsa_build_block_mask_workspace_bytes(int B, int H, int N, int d
  * (row stride NB, ascending, each in [0,NB)).  Every list needs at least one entry; a malformed
  * entry sets AVSA_ERR_BAD_MASK in the status record and that block is skipped without any
  * out-of-range access.  o is bf16 with the strides of q; lse (optional) is fp32 [B,H,N] natural log.
+ *
+ * Two kernels run: a fast one that keeps each row's first-tile maximum as the softmax reference (no
+ * rescaling of the accumulator), and behind it the exact-rescaling kernel for the work items the fast
+ * one had to give up (a row whose sum of exp(logit - reference) ends above 2^64 or is not finite; values of
+ * v are assumed to stay below 2^60 in magnitude).
+ * After the call ws holds, behind its first AVSA_STATUS_BYTES bytes, one int32 per (b,h,query block):
+ * 1 where the item was recomputed by the exact kernel, else 0 (diagnostic; results do not depend on it).
  */
 AVSA_API int avsa_sparse_self_attn(int B, int H, int N, int d, int blk, avsa_bf16_4d q, avsa_bf16_4d k, avsa_bf16_4d v,
                           const int32_t* col_idx, const int32_t* col_cnt, void* o_bf16, float* lse,

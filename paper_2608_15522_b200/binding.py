@@ -143,6 +143,9 @@ def _check(status: int, where: str) -> None:
         raise AvsaError(status, where)
 
 
+AVSA_STATUS_BYTES = 256
+
+
 def avsa_read_status(ws: torch.Tensor) -> Tuple[int, Tuple[int, int, int]]:
     """Synchronises the current stream and returns (status, (where, item, aux)) of a workspace."""
     detail = (ctypes.c_int * 3)()

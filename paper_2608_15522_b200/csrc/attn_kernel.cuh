@@ -59,6 +59,7 @@ struct AttnParams {
   int n_split, tiles_per_split;
   // both
   StatusRecord* status;
+  const int* redo_flags;    // optional [items]: run only the work items flagged by the fast kernel
   int H;
   int Nq, NQT;              // query rows and query tiles
   int Nk, NKB;              // key rows and key tiles
@@ -107,6 +108,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__
     cnt = min(p.NKB, kb0 + p.tiles_per_split) - kb0;
   }
   const int item = ((b * p.H + h) * p.NQT + qt) * (kListIn ? 1 : p.n_split) + split;
+  if (p.redo_flags != nullptr && p.redo_flags[item] == 0) return;   // already computed by the fast kernel
 
   // ---- validation: nothing is loaded through a bad list entry
   {

@@ -1,23 +1,34 @@
 // avsa_sparse_self_attn: block-sparse video self-attention under the protected block mask
 // (Eq. 10 / Eq. 11; Eq. 5 when every list is full).  Host side: argument checks, tensor maps, launch.
-#include "attn_kernel.cuh"
+#include "attn_fast_kernel.cuh"
 
 namespace avsa {
 
 template <int BLK, int D>
 static int launch_sparse_attn(int B, int H, int N, const avsa_bf16_4d& q, const avsa_bf16_4d& k,
-                              const avsa_bf16_4d& v, void* o, const AttnParams& prm, cudaStream_t st) {
+                              const avsa_bf16_4d& v, void* o, const AttnParams& prm, int* redo, cudaStream_t st) {
   using L = AttnSmem<BLK, D>;
   CUtensorMap tq, tk, tv, to;
   if (!encode_bf16_tile_map(&tq, q.ptr, B, H, N, D, q.stride_b, q.stride_h, q.stride_n, BLK)) return AVSA_ERR_CUDA;
   if (!encode_bf16_tile_map(&tk, k.ptr, B, H, N, D, k.stride_b, k.stride_h, k.stride_n, BLK)) return AVSA_ERR_CUDA;
   if (!encode_bf16_tile_map(&tv, v.ptr, B, H, N, D, v.stride_b, v.stride_h, v.stride_n, BLK)) return AVSA_ERR_CUDA;
   if (!encode_bf16_tile_map(&to, o, B, H, N, D, q.stride_b, q.stride_h, q.stride_n, BLK)) return AVSA_ERR_CUDA;
+  using LF = FastSmem<BLK, D>;
+  if (cudaFuncSetAttribute(attn_fast_kernel<BLK, D, MODE_LIST>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           LF::kTotal) != cudaSuccess)
+    return AVSA_ERR_CUDA;
   if (cudaFuncSetAttribute(attn_fwd_kernel<BLK, D, MODE_LIST>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            L::kTotal) != cudaSuccess)
     return AVSA_ERR_CUDA;
   dim3 grid(prm.NQT, H, B);
-  attn_fwd_kernel<BLK, D, MODE_LIST><<<grid, kAttnThreads, L::kTotal, st>>>(tq, tk, tv, to, prm);
+  // Fast kernel first; it flags the (rare) work items whose logits outgrow its fixed reference maxima, and the
+  // exact-rescaling kernel behind it recomputes exactly those (its other CTAs return at once).
+  AttnParams fast = prm;
+  fast.redo_flags = nullptr;
+  attn_fast_kernel<BLK, D, MODE_LIST><<<grid, kAttnThreads, LF::kTotal, st>>>(tq, tk, tv, to, fast, redo);
+  AttnParams exact = prm;
+  exact.redo_flags = redo;
+  attn_fwd_kernel<BLK, D, MODE_LIST><<<grid, kAttnThreads, L::kTotal, st>>>(tq, tk, tv, to, exact);
   return cudaGetLastError() == cudaSuccess ? AVSA_OK : AVSA_ERR_CUDA;
 }
 
@@ -35,7 +46,8 @@ extern "C" __attribute__((visibility("default"))) void avsa_debug_set_trace(long
 
 extern "C" size_t avsa_sparse_self_attn_workspace_bytes(int B, int H, int N, int d, int blk) {
   if (B <= 0 || H <= 0 || N <= 0 || d <= 0 || blk <= 0) return 0;
-  return kStatusBytes;
+  const size_t nb = (static_cast<size_t>(N) + blk - 1) / blk;
+  return kStatusBytes + align_up(static_cast<size_t>(B) * H * nb * sizeof(int), 256);   // status + one flag per item
 }
 
 extern "C" int avsa_sparse_self_attn(int B, int H, int N, int d, int blk, avsa_bf16_4d q, avsa_bf16_4d k,
@@ -47,7 +59,7 @@ extern "C" int avsa_sparse_self_attn(int B, int H, int N, int d, int blk, avsa_b
   if (!tensor_ok(q, B, H) || !tensor_ok(k, B, H) || !tensor_ok(v, B, H)) return AVSA_ERR_INVALID_ARG;
   if (col_idx == nullptr || col_cnt == nullptr || o_bf16 == nullptr || !aligned16(o_bf16)) return AVSA_ERR_INVALID_ARG;
   if (softmax_scale < 0.f || softmax_scale != softmax_scale) return AVSA_ERR_INVALID_ARG;
-  if (ws == nullptr || ws_bytes < kStatusBytes) return AVSA_ERR_WORKSPACE;
+  if (ws == nullptr || ws_bytes < avsa_sparse_self_attn_workspace_bytes(B, H, N, d, blk)) return AVSA_ERR_WORKSPACE;
   if (!device_is_sm100()) return AVSA_ERR_UNSUPPORTED;
   cudaStream_t st = as_stream(stream);
   AttnParams prm = {};
@@ -65,6 +77,7 @@ extern "C" int avsa_sparse_self_attn(int B, int H, int N, int d, int blk, avsa_b
   prm.trace = g_trace_buffer;
 #endif
   clear_status_kernel<<<1, 1, 0, st>>>(prm.status);
-  if (d == 128) return launch_sparse_attn<128, 128>(B, H, N, q, k, v, o_bf16, prm, st);
-  return launch_sparse_attn<64, 64>(B, H, N, q, k, v, o_bf16, prm, st);
+  int* redo = reinterpret_cast<int*>(static_cast<uint8_t*>(ws) + kStatusBytes);
+  if (d == 128) return launch_sparse_attn<128, 128>(B, H, N, q, k, v, o_bf16, prm, redo, st);
+  return launch_sparse_attn<64, 64>(B, H, N, q, k, v, o_bf16, prm, redo, st);
 }

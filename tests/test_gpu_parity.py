@@ -208,6 +208,43 @@ def test_sparse_attention_single_and_odd_counts():
     _run_sparse_case(w, 3, idx, cnt)
 
 
+@pytest.mark.parametrize("step,expect_redo", [(1.0, False), (16.0, True)])
+def test_sparse_attention_row_maxima_growing_along_the_key_axis(step, expect_redo):
+    """Logits that grow from key block to key block.  The fast kernel keeps the first tile's row maximum
+    as its reference: a moderate growth stays inside its headroom, a steep one makes it hand the work item
+    to the exact-rescaling kernel (flag words behind the status record in the workspace).  Both must match
+    the oracle; in the steep case the flags must actually have been raised."""
+    w = wl.WORKLOADS["medium128"]
+    q, k, v = wl.make_self_qkv(w, 6)
+    NB = w.n_blocks
+    u = 1.0 / np.sqrt(w.d)
+    q = (q.float() + 8.0 * u).to(torch.bfloat16)
+    ramp = torch.arange(w.n_video, dtype=torch.float32).div(w.blk, rounding_mode="floor") * step
+    k = (k.float() + (ramp * u).view(1, 1, -1, 1)).to(torch.bfloat16)
+    rng = np.random.default_rng(8)
+    idx = np.full((w.B, w.H, NB, NB), -1, np.int32)
+    cnt = np.zeros((w.B, w.H, NB), np.int32)
+    for b in range(w.B):
+        for h in range(w.H):
+            for i in range(NB):
+                c = NB if i % 4 == 0 else 1 + int(rng.integers(NB))
+                cols = np.sort(rng.choice(NB, size=c, replace=False))
+                idx[b, h, i, :c] = cols
+                cnt[b, h, i] = c
+    o, lse, ws = av.avsa_sparse_self_attn(q.cuda(), k.cuda(), v.cuda(), torch.from_numpy(idx).cuda(),
+                                          torch.from_numpy(cnt).cuda(), w.blk, want_lse=True)
+    _status_ok(ws)
+    want_o, want_l = orc.masked_attention(_np64(q), _np64(k), _np64(v), idx, cnt, w.blk)
+    _close(_np64(o), want_o, "growing maxima O")
+    _close(_np64(lse), want_l, "growing maxima lse")
+    flags = ws[av.AVSA_STATUS_BYTES:av.AVSA_STATUS_BYTES + 4 * w.B * w.H * NB].view(torch.int32).cpu().numpy()
+    assert set(np.unique(flags)) <= {0, 1}
+    assert (flags.sum() > 0) == expect_redo
+    if expect_redo:
+        # items with a single key block never outgrow their reference
+        assert np.all(flags.reshape(w.B, w.H, NB)[cnt == 1] == 0)
+
+
 def test_sparse_attention_strided_bnhd_layout():
     w = wl.WORKLOADS["small128"]
     q, k, v = wl.make_self_qkv(w, 4)
