@@ -128,8 +128,9 @@ AVSA_API size_t avsa_build_block_mask_workspace_bytes(int B, int H, int N, int d
  * rescaling of the accumulator), and behind it the exact-rescaling kernel for the work items the fast
  * one had to give up (a row whose sum of exp(logit - reference) ends above 2^64 or is not finite; values of
  * v are assumed to stay below 2^60 in magnitude).
- * After the call ws holds, behind its first AVSA_STATUS_BYTES bytes, one int32 per (b,h,query block):
- * 1 where the item was recomputed by the exact kernel, else 0 (diagnostic; results do not depend on it).
+ * After the call the int32 at byte 16 of ws is the number of work items the exact kernel recomputed, and
+ * their indices ((b*H + h)*NB + query block, in no particular order) follow as int32 behind the first
+ * AVSA_STATUS_BYTES bytes (diagnostic; results do not depend on it).
  */
 AVSA_API int avsa_sparse_self_attn(int B, int H, int N, int d, int blk, avsa_bf16_4d q, avsa_bf16_4d k, avsa_bf16_4d v,
                           const int32_t* col_idx, const int32_t* col_cnt, void* o_bf16, float* lse,

@@ -269,6 +269,15 @@ def avsa_sparse_self_attn(q, k, v, col_idx, col_cnt, blk, softmax_scale=0.0, wan
     return o, lse, ws
 
 
+def avsa_sparse_self_attn_redo_items(ws: torch.Tensor):
+    """Diagnostic: (count, int32 array) of the work items ((b*H + h)*NB + query block) that the last
+    avsa_sparse_self_attn call on this workspace recomputed with the exact-rescaling kernel."""
+    torch.cuda.synchronize(ws.device)
+    n = int(ws[16:20].view(torch.int32).item())
+    items = ws[AVSA_STATUS_BYTES:AVSA_STATUS_BYTES + 4 * n].view(torch.int32).cpu().numpy()
+    return n, items
+
+
 def avsa_protected_rows_attn_workspace_bytes(B, H, N, d, blk, n_protect) -> int:
     return int(load_library().avsa_protected_rows_attn_workspace_bytes(B, H, N, d, blk, n_protect))
 

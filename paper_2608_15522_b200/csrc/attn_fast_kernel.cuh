@@ -15,9 +15,9 @@
 //     only at the first store of the new P;
 //   * two warps issue MMAs, one the Q K^T products and one the P V products: every MMA and every barrier
 //     wait costs the issuing thread tens of cycles, which one warp doing both would serialise.
-// A row whose sum, relative to m_ref, ends above 2^64 (or not finite) outgrew its reference: the CTA marks
-// its work item in `redo_flags`, and attn_fwd_kernel (launched behind this kernel, its CTAs return at once
-// unless flagged) recomputes the item with exact rescaling.  Unflagged items get redo_flags = 0.
+// A row whose sum, relative to m_ref, ends above 2^64 (or not finite) outgrew its reference: the CTA appends
+// its work item to `redo_list` (count in the status record), and attn_redo_kernel, a small grid launched
+// behind this kernel, recomputes the listed items with exact rescaling.
 //
 // Producer warps, shared-memory rings, list validation and bounded waits are as in attn_fwd_kernel.
 #pragma once
@@ -53,7 +53,7 @@ template <int BLK, int D, int MODE>
 __global__ void __launch_bounds__(kAttnThreads, 1)
 attn_fast_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUtensorMap tmk,
                  const __grid_constant__ CUtensorMap tmv, const __grid_constant__ CUtensorMap tmo,
-                 const AttnParams p, int* __restrict__ redo_flags) {
+                 const AttnParams p, int* __restrict__ redo_list) {
   using L = FastSmem<BLK, D>;
   constexpr bool kListIn = (MODE == MODE_LIST);
   constexpr bool kDirectOut = (MODE != MODE_RANGE);
@@ -94,12 +94,10 @@ attn_fast_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant_
     if (misaligned) bad = 1;
     const int any_bad = __syncthreads_or(bad);
     if (any_bad) {
-      if (tid == 0) {
+      if (tid == 0)
         report_status(p.status, misaligned ? AVSA_ERR_CUDA : AVSA_ERR_BAD_MASK, misaligned ? kWhereSmemAlign : kWhereList,
                       item, cnt);
-        redo_flags[item] = 0;     // nothing to recompute: the item is refused, not deferred
-      }
-      return;
+      return;     // nothing to recompute: the item is refused, not deferred
     }
   }
 
@@ -487,7 +485,7 @@ attn_fast_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant_
   }
   tc_fence_before();
   __syncthreads();
-  if (tid == 0) redo_flags[item] = (misc[2] != 0u) ? 1 : 0;
+  if (tid == 0 && misc[2] != 0u) redo_list[atomicAdd(&p.status->redo_count, 1)] = item;
   if (warp == 2) tmem_dealloc(tmem, 512);
 }
 

@@ -59,7 +59,6 @@ struct AttnParams {
   int n_split, tiles_per_split;
   // both
   StatusRecord* status;
-  const int* redo_flags;    // optional [items]: run only the work items flagged by the fast kernel
   int H;
   int Nq, NQT;              // query rows and query tiles
   int Nk, NKB;              // key rows and key tiles
@@ -79,11 +78,12 @@ struct AttnParams {
 #define AVSA_STAMP(role, tile, slot) do { } while (0)
 #endif
 
+// One work item of the tile kernel: query tile `bx` (MODE_LIST) or query tile / key split `bx`
+// (range modes) of head `by`, batch item `bz`.  Called once per CTA by attn_fwd_kernel and once per
+// flagged work item by attn_redo_kernel; every thread of the CTA must call it.
 template <int BLK, int D, int MODE>
-__global__ void __launch_bounds__(kAttnThreads, 1)
-attn_fwd_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUtensorMap tmk,
-                const __grid_constant__ CUtensorMap tmv, const __grid_constant__ CUtensorMap tmo,
-                const AttnParams p) {
+__device__ __forceinline__ void attn_fwd_body(const CUtensorMap* tmq, const CUtensorMap* tmk, const CUtensorMap* tmv,
+                                              const CUtensorMap* tmo, const AttnParams& p, int bx, int by, int bz) {
   using L = AttnSmem<BLK, D>;
   constexpr bool kListIn = (MODE == MODE_LIST);          // explicit list of key tiles (else a contiguous range)
   constexpr bool kDirectOut = (MODE != MODE_RANGE);      // final bf16 tile + LSE (else a partial result)
@@ -93,23 +93,21 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__
   extern __shared__ __align__(1024) uint8_t smem[];
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int h = blockIdx.y, b = blockIdx.z;
+  const int h = by, b = bz;
   int qt, split = 0, kb0 = 0, cnt;
   const int32_t* list = nullptr;
   if (kListIn) {
-    qt = blockIdx.x;
+    qt = bx;
     const int row_id = (b * p.H + h) * p.NQT + qt;
     list = p.col_idx + static_cast<int64_t>(row_id) * p.NKB;
     cnt = p.col_cnt[row_id];
   } else {
-    qt = blockIdx.x / p.n_split;
-    split = blockIdx.x % p.n_split;
+    qt = bx / p.n_split;
+    split = bx % p.n_split;
     kb0 = split * p.tiles_per_split;
     cnt = min(p.NKB, kb0 + p.tiles_per_split) - kb0;
   }
   const int item = ((b * p.H + h) * p.NQT + qt) * (kListIn ? 1 : p.n_split) + split;
-  if (p.redo_flags != nullptr && p.redo_flags[item] == 0) return;   // already computed by the fast kernel
-
   // ---- validation: nothing is loaded through a bad list entry
   {
     int bad = (cnt < 1 || cnt > p.NKB) ? 1 : 0;
@@ -156,14 +154,15 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__
     mbar_init(BAR(FINAL), 1);
     misc[1] = 0u;
     fence_mbar_init();
-    prefetch_tmap(&tmq);
-    prefetch_tmap(&tmk);
-    prefetch_tmap(&tmv);
-    if (kDirectOut) prefetch_tmap(&tmo);
+    prefetch_tmap(tmq);
+    prefetch_tmap(tmk);
+    prefetch_tmap(tmv);
+    if (kDirectOut) prefetch_tmap(tmo);
   }
   if (warp == 2) {
+    // (the allocation permit is kept: attn_redo_kernel runs this body several times in one CTA, and with one
+    // CTA per SM nobody else is waiting for it)
     tmem_alloc(smem_u32(smem + L::kMisc), 512);
-    tmem_relinquish();
   }
   tc_fence_before();
   __syncthreads();
@@ -192,13 +191,13 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__
     // ------------------------------------------------------------------ TMA producers: warp 0 K (and Q), warp 3 V
     asm volatile("setmaxnreg.dec.sync.aligned.u32 64;");
     const bool is_k = (warp == 0);
-    const CUtensorMap* tm = is_k ? &tmk : &tmv;
+    const CUtensorMap* tm = is_k ? tmk : tmv;
     const int FULL = is_k ? K_FULL : V_FULL, EMPTY = is_k ? K_EMPTY : V_EMPTY;
     const uint32_t base = smem_u32(smem + (is_k ? L::kK : L::kV));
     if (is_k && lane == 0) {
       mbar_expect_tx(BAR(Q_FULL), BLK * D * 2);
       for (int pn = 0; pn < NPANEL; pn++)
-        tma_load_4d(smem_u32(smem + L::kQ) + pn * QPANEL_BYTES, &tmq, BAR(Q_FULL), pn * 64, qt * BLK, h, b);
+        tma_load_4d(smem_u32(smem + L::kQ) + pn * QPANEL_BYTES, tmq, BAR(Q_FULL), pn * 64, qt * BLK, h, b);
     }
     int s = 0, fpar = 0;     // stage, and the parity of the "empty" phase to wait for once the ring has wrapped
     for (int t0 = 0; t0 < cnt; t0 += 32) {
@@ -473,7 +472,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__
     asm volatile("bar.sync 1, 256;" ::: "memory");
     if (kDirectOut && ok && warp == 4 && lane == 0) {
       for (int pn = 0; pn < NPANEL; pn++)
-        tma_store_4d(&tmo, smem_u32(smem + L::kQ) + pn * QPANEL_BYTES, pn * 64, qt * BLK, h, b);
+        tma_store_4d(tmo, smem_u32(smem + L::kQ) + pn * QPANEL_BYTES, pn * 64, qt * BLK, h, b);
       tma_store_commit();
       tma_store_wait_read();
     }
@@ -481,6 +480,43 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__
   tc_fence_before();
   __syncthreads();
   if (warp == 2) tmem_dealloc(tmem, 512);
+}
+
+template <int BLK, int D, int MODE>
+__global__ void __launch_bounds__(kAttnThreads, 1)
+attn_fwd_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUtensorMap tmk,
+                const __grid_constant__ CUtensorMap tmv, const __grid_constant__ CUtensorMap tmo,
+                const AttnParams p) {
+  attn_fwd_body<BLK, D, MODE>(&tmq, &tmk, &tmv, &tmo, p, blockIdx.x, blockIdx.y, blockIdx.z);
+}
+
+// Exact-rescaling pass behind attn_fast_kernel: recomputes the work items that kernel listed (normally
+// none: then every CTA of this small grid returns at once).  CTA c takes entries c, c + gridDim.x, ...
+template <int BLK, int D>
+__global__ void __launch_bounds__(kAttnThreads, 1)
+attn_redo_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUtensorMap tmk,
+                 const __grid_constant__ CUtensorMap tmv, const __grid_constant__ CUtensorMap tmo,
+                 const AttnParams p, const int* __restrict__ redo_list) {
+  using L = AttnSmem<BLK, D>;
+  extern __shared__ __align__(1024) uint8_t smem[];
+  const int n_redo = p.status->redo_count;
+  const int warp = threadIdx.x >> 5;
+  for (int k = blockIdx.x; k < n_redo; k += gridDim.x) {
+    const int item = redo_list[k];                     // (b * H + h) * NQT + qt
+    const int qt = item % p.NQT, bh = item / p.NQT;
+    attn_fwd_body<BLK, D, MODE_LIST>(&tmq, &tmk, &tmv, &tmo, p, qt, bh % p.H, bh / p.H);
+    // back to the launch state for the next item: every warp at the launch register count, barriers invalidated
+    if (warp < 4) {
+      asm volatile("setmaxnreg.inc.sync.aligned.u32 168;");
+    } else {
+      asm volatile("setmaxnreg.dec.sync.aligned.u32 168;");
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      for (int i = 0; i < L::kNumBars; i++) mbar_inval(smem_u32(smem + L::kBars) + i * 8);
+    }
+    __syncthreads();
+  }
 }
 
 // ------------------------------------------------------------------------------------------------

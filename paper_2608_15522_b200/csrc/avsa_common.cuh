@@ -16,6 +16,7 @@ struct StatusRecord {
   int where;      // which wait / check
   int item;       // work item (block index)
   int aux;        // tile index or offending value
+  int redo_count; // sparse attention: work items the fast kernel left to the exact kernel in this call
 };
 constexpr size_t kStatusBytes = 256;   // the record, padded so that what follows stays 256-byte aligned
 
@@ -33,6 +34,7 @@ static __global__ void clear_status_kernel(StatusRecord* st) {
   st->where = 0;
   st->item = 0;
   st->aux = 0;
+  st->redo_count = 0;
 }
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }

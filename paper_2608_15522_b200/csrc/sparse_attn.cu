@@ -17,18 +17,16 @@ static int launch_sparse_attn(int B, int H, int N, const avsa_bf16_4d& q, const 
   if (cudaFuncSetAttribute(attn_fast_kernel<BLK, D, MODE_LIST>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            LF::kTotal) != cudaSuccess)
     return AVSA_ERR_CUDA;
-  if (cudaFuncSetAttribute(attn_fwd_kernel<BLK, D, MODE_LIST>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           L::kTotal) != cudaSuccess)
+  if (cudaFuncSetAttribute(attn_redo_kernel<BLK, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal) !=
+      cudaSuccess)
     return AVSA_ERR_CUDA;
   dim3 grid(prm.NQT, H, B);
-  // Fast kernel first; it flags the (rare) work items whose logits outgrow its fixed reference maxima, and the
-  // exact-rescaling kernel behind it recomputes exactly those (its other CTAs return at once).
-  AttnParams fast = prm;
-  fast.redo_flags = nullptr;
-  attn_fast_kernel<BLK, D, MODE_LIST><<<grid, kAttnThreads, LF::kTotal, st>>>(tq, tk, tv, to, fast, redo);
-  AttnParams exact = prm;
-  exact.redo_flags = redo;
-  attn_fwd_kernel<BLK, D, MODE_LIST><<<grid, kAttnThreads, L::kTotal, st>>>(tq, tk, tv, to, exact);
+  // Fast kernel first; it lists the (rare) work items whose rows outgrow its fixed reference maxima, and the
+  // exact-rescaling kernel behind it recomputes exactly those.
+  attn_fast_kernel<BLK, D, MODE_LIST><<<grid, kAttnThreads, LF::kTotal, st>>>(tq, tk, tv, to, prm, redo);
+  const long long items = static_cast<long long>(prm.NQT) * H * B;
+  const int redo_grid = static_cast<int>(items < 148 ? items : 148);
+  attn_redo_kernel<BLK, D><<<redo_grid, kAttnThreads, L::kTotal, st>>>(tq, tk, tv, to, prm, redo);
   return cudaGetLastError() == cudaSuccess ? AVSA_OK : AVSA_ERR_CUDA;
 }
 
