@@ -35,9 +35,9 @@ UNIT = "TFLOP/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the sparse attention kernel, from the ncu capture
 # summarised under profiles/ (None until a capture exists for that workload)
-NCU_TRAFFIC_BYTES = {"mid": 428.3e6,      # captured (profiles/attn_fwd_kernel_mid.md)
-                     "ovi": 785.8e6}      # the mid capture scaled by Q+K+V+O bytes: too large to capture under the size rule
-KERNELS_PER_STEP = 12   # cross: clear, pass 1, merge, pass 2, head sum; mask: select, pool, scores, rows; attn: clear, fast, exact
+NCU_TRAFFIC_BYTES = {"mid": 427.3e6,      # captured (profiles/attn_fast_kernel_mid.md)
+                     "ovi": 784.0e6}      # the mid capture scaled by Q+K+V+O bytes: too large to capture under the size rule
+KERNELS_PER_STEP = 12   # cross: clear, pass 1, merge, pass 2, head sum; mask: select, pool, scores, rows; attn: clear, fast, redo
 
 
 def load_peaks():
