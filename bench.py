@@ -236,6 +236,8 @@ def run_ours(args, w):
     t_cross = float(np.mean([e[0].elapsed_time(e[1]) for e in ev]))
     t_mask = float(np.mean([e[1].elapsed_time(e[2]) for e in ev]))
     t_attn = float(np.mean([e[2].elapsed_time(e[3]) for e in ev]))
+    step_ms = [e[0].elapsed_time(e[3]) for e in ev]
+    attn_ms = [e[2].elapsed_time(e[3]) for e in ev]
     clocks = sampler.stop() if sampler else None
 
     # ---- dense baselines on the same tensors (outside the timed region)
@@ -373,7 +375,9 @@ def run_ours(args, w):
                        "l2": "inputs (Q,K,V of both attentions, 1.2 GB) are larger than the 126 MB L2; no flush",
                        "multi_gpu": "independent replica per GPU, no data-path collective"},
             "ms": {"cross_attn_scores": t_cross, "build_block_mask": t_mask, "sparse_self_attn": t_attn,
-                   "dense_keep_all_ours": t_dense_ours, "dense_library_sdpa": t_dense_lib},
+                   "dense_keep_all_ours": t_dense_ours, "dense_library_sdpa": t_dense_lib,
+                   "step_median": float(np.median(step_ms)), "step_min": float(np.min(step_ms)),
+                   "sparse_self_attn_median": float(np.median(attn_ms)), "sparse_self_attn_min": float(np.min(attn_ms))},
             "speedup_vs_dense": {"attn_only": dense_best / t_attn, "layer_step": dense_best / ms_per_step,
                                  "dense_is": "library_sdpa" if dense_best == t_dense_lib else "keep_all_ours"},
             "token_exact_protection": {
