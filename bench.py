@@ -372,6 +372,10 @@ def run_ours(args, w):
                        "blk": w.blk, "keep_pct": w.keep_pct, "protect_pct": w.protect_pct, "k_keep": k_keep,
                        "n_protect": n_protect, "protected_blocks": prot_blocks, "n_blocks": NB,
                        "executed_pair_fraction": pairs / float(w.B * w.H * NB * NB),
+                       # Eq. 16 beside it: kappa + rho on tokens, and kappa + p_b (1 - kappa) with p_b the
+                       # protected-BLOCK fraction (what block-level protection can reach at best)
+                       "eq16_kappa_plus_rho": (w.keep_pct + w.protect_pct) / 100.0,
+                       "eq16_kappa_plus_pb": k_keep / float(NB) + prot_blocks / float(w.B * NB) * (1.0 - k_keep / float(NB)),
                        "l2": "inputs (Q,K,V of both attentions, 1.2 GB) are larger than the 126 MB L2; no flush",
                        "multi_gpu": "independent replica per GPU, no data-path collective"},
             "ms": {"cross_attn_scores": t_cross, "build_block_mask": t_mask, "sparse_self_attn": t_attn,
@@ -394,7 +398,7 @@ def run_ours(args, w):
                                  "note": "Eq. 12-15 on [B,N,H*d] feature maps; reads both maps once; L2 not flushed "
                                          "between repetitions but the 406 MB exceed it"},
             "executed_tflops": achieved,
-            "roofline": {"kernel": "attn_fast_kernel<128,128,MODE_LIST> (avsa_sparse_self_attn)", "bound": "tensor",
+            "roofline": {"kernel": "attn_fast_kernel<128,128> (avsa_sparse_self_attn)", "bound": "tensor",
                          "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
                          "peak_source": f"{peak_kind} bf16_tflops (burst)", "frac_of_sustained": achieved / sustained,
                          "frac_of_nominal_2250": achieved / 2250.0,

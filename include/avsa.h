@@ -67,6 +67,11 @@ typedef struct {
 #define AVSA_PROTECT_TOKENS 8u          /* lists carry the base pattern only (no block is made dense); the
                                            protected rows are restored by avsa_protected_rows_attn */
 
+/* Optional, ORed into flags: a block counts as protected only if it holds at least n (1..blk) protected tokens.
+ * Not in the paper: in raster order a compact region straddles many blocks, and n > 1 trades the protection of
+ * stray tokens for fewer dense blocks.  n = 0 or 1 is the block lift of Eq. 9 (any protected token). */
+#define AVSA_MIN_TOKENS_PER_BLOCK(n) (((unsigned)(n) & 0xffu) << 8)
+
 /*
  * (1) Cross-attention with response scores -- Eq. 1, Eq. 2 (and the running blend of Eq. 4).
  *

@@ -95,16 +95,20 @@ def protected_tokens(s, n_protect):
     return flags
 
 
-def protected_blocks(prot_tok, blk):
-    """A block is protected iff any of its tokens is (block lift of Eq. 9).  -> uint8 [B,NB]."""
+def protected_blocks(prot_tok, blk, min_tokens=1):
+    """A block is protected iff it holds at least ``min_tokens`` protected tokens; with the default 1 this
+    is the block lift of Eq. 9 (any protected token).  -> uint8 [B,NB]."""
     prot_tok = np.asarray(prot_tok)
     B, N = prot_tok.shape
     nb = (N + blk - 1) // blk
     out = np.zeros((B, nb), np.uint8)
     for b in range(B):
+        count = [0] * nb
         for i in range(N):
             if prot_tok[b, i]:
-                out[b, i // blk] = 1
+                count[i // blk] += 1
+        for j in range(nb):
+            out[b, j] = 1 if count[j] >= max(1, min_tokens) else 0
     return out
 
 
@@ -176,7 +180,8 @@ def keep_to_lists(keep):
     return idx, cnt
 
 
-def build_block_mask(bs, scores, n_protect, k_keep, blk, n_tokens, protect_rows=True, protect_cols=False):
+def build_block_mask(bs, scores, n_protect, k_keep, blk, n_tokens, protect_rows=True, protect_cols=False,
+                     min_tokens=1):
     """Block scores + token scores -> (col_idx, col_cnt, prot_tok, prot_blk), the whole mask step."""
     bs = np.asarray(bs)
     B = bs.shape[0]
@@ -184,7 +189,7 @@ def build_block_mask(bs, scores, n_protect, k_keep, blk, n_tokens, protect_rows=
         prot_tok = protected_tokens(scores, n_protect)
     else:
         prot_tok = np.zeros((B, n_tokens), np.uint8)
-    prot_blk = protected_blocks(prot_tok, blk)
+    prot_blk = protected_blocks(prot_tok, blk, min_tokens)
     keep = apply_protection(topk_blocks(bs, k_keep), prot_blk, protect_rows, protect_cols)
     idx, cnt = keep_to_lists(keep)
     return idx, cnt, prot_tok, prot_blk

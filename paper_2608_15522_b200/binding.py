@@ -28,6 +28,12 @@ AVSA_PROTECT_COLS = 2
 AVSA_USE_GIVEN_BLOCK_SCORES = 4
 AVSA_PROTECT_TOKENS = 8
 
+
+def AVSA_MIN_TOKENS_PER_BLOCK(n: int) -> int:
+    """Flag bits: a block is protected only if it holds at least n protected tokens."""
+    return (int(n) & 0xFF) << 8
+
+
 EXPORTS = (
     "avsa_cross_attn_scores", "avsa_cross_attn_scores_workspace_bytes",
     "avsa_build_block_mask", "avsa_build_block_mask_workspace_bytes", "avsa_build_block_mask_static",

@@ -49,14 +49,13 @@ struct FastSmem {
 
 enum FastWhere { kFastSFree = 61, kFastPFree, kFastMref };
 
-template <int BLK, int D, int MODE>
+// List mode only (the block-sparse self-attention call); the range modes stay with attn_fwd_kernel.
+template <int BLK, int D>
 __global__ void __launch_bounds__(kAttnThreads, 1)
 attn_fast_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUtensorMap tmk,
                  const __grid_constant__ CUtensorMap tmv, const __grid_constant__ CUtensorMap tmo,
                  const AttnParams p, int* __restrict__ redo_list) {
   using L = FastSmem<BLK, D>;
-  constexpr bool kListIn = (MODE == MODE_LIST);
-  constexpr bool kDirectOut = (MODE != MODE_RANGE);
   constexpr int NPANEL = D / 64;
   constexpr int PANEL_BYTES = BLK * 128;
   constexpr int QPANEL_BYTES = 128 * 128;
@@ -64,31 +63,19 @@ attn_fast_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant_
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int h = blockIdx.y, b = blockIdx.z;
-  int qt, split = 0, kb0 = 0, cnt;
-  const int32_t* list = nullptr;
-  if (kListIn) {
-    qt = blockIdx.x;
-    const int row_id = (b * p.H + h) * p.NQT + qt;
-    list = p.col_idx + static_cast<int64_t>(row_id) * p.NKB;
-    cnt = p.col_cnt[row_id];
-  } else {
-    qt = blockIdx.x / p.n_split;
-    split = blockIdx.x % p.n_split;
-    kb0 = split * p.tiles_per_split;
-    cnt = min(p.NKB, kb0 + p.tiles_per_split) - kb0;
-  }
-  const int item = ((b * p.H + h) * p.NQT + qt) * (kListIn ? 1 : p.n_split) + split;
+  const int qt = blockIdx.x;
+  const int item = (b * p.H + h) * p.NQT + qt;
+  const int32_t* list = p.col_idx + static_cast<int64_t>(item) * p.NKB;
+  const int cnt = p.col_cnt[item];
 
   // ---- validation: nothing is loaded through a bad list entry (the fallback kernel reports it too)
   {
     int bad = (cnt < 1 || cnt > p.NKB) ? 1 : 0;
-    if (kListIn) {
-      const int n = min(max(cnt, 0), p.NKB);
-      for (int t = tid; t < n; t += kAttnThreads) {
-        const int kb = list[t];
-        const int prev = t > 0 ? list[t - 1] : -1;
-        if (kb < 0 || kb >= p.NKB || kb <= prev) bad = 1;
-      }
+    const int n = min(max(cnt, 0), p.NKB);
+    for (int t = tid; t < n; t += kAttnThreads) {
+      const int kb = list[t];
+      const int prev = t > 0 ? list[t - 1] : -1;
+      if (kb < 0 || kb >= p.NKB || kb <= prev) bad = 1;
     }
     const bool misaligned = (smem_u32(smem) & 1023u) != 0u;
     if (misaligned) bad = 1;
@@ -138,7 +125,7 @@ attn_fast_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant_
     prefetch_tmap(&tmq);
     prefetch_tmap(&tmk);
     prefetch_tmap(&tmv);
-    if (kDirectOut) prefetch_tmap(&tmo);
+    prefetch_tmap(&tmo);
   }
   if (warp == 2) {
     tmem_alloc(smem_u32(smem + L::kMisc), 512);
@@ -179,8 +166,7 @@ attn_fast_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant_
     int s = 0, fpar = 0;
     int issued = 0;          // lane 0: number of tiles whose load has been issued
     for (int t0 = 0; t0 < cnt; t0 += 32) {
-      int mine = kb0 + t0 + lane;
-      if (kListIn) mine = (t0 + lane < cnt) ? list[t0 + lane] : 0;
+      const int mine = (t0 + lane < cnt) ? list[t0 + lane] : 0;
       const int nn = min(32, cnt - t0);
       for (int j = 0; j < nn; j++) {
         const int kb = __shfl_sync(0xffffffffu, mine, j);
@@ -323,7 +309,7 @@ attn_fast_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant_
     const int w = (warp - 4) >> 2;               // group
     const int row = ((warp & 3) << 5) + lane;    // row of the tile == TMEM lane
     const uint32_t lane_off = static_cast<uint32_t>((warp & 3) * 32) << 16;
-    const int last_kb = kListIn ? list[cnt - 1] : kb0 + cnt - 1;
+    const int last_kb = list[cnt - 1];
     const int ragged_valid = (last_kb == p.NKB - 1) ? (p.Nk - last_kb * BLK) : BLK;
     float m_ref = 0.f, l_run = 0.f;
     uint64_t sum2[4] = {0ull, 0ull, 0ull, 0ull};
@@ -444,39 +430,26 @@ attn_fast_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant_
 #pragma unroll
         for (int j = 0; j < 32; j++) v[j] = __uint_as_float(o0[j]) * inv;
         if (row < BLK) {
-          if (kDirectOut) {
 #pragma unroll
-            for (int g = 0; g < 4; g++) {
-              const int col = col0 + g * 8;
-              const int panel = col >> 6, chunk = (col & 63) >> 3;
-              uint4 val;
-              val.x = pack_bf16x2(v[g * 8 + 0], v[g * 8 + 1]);
-              val.y = pack_bf16x2(v[g * 8 + 2], v[g * 8 + 3]);
-              val.z = pack_bf16x2(v[g * 8 + 4], v[g * 8 + 5]);
-              val.w = pack_bf16x2(v[g * 8 + 6], v[g * 8 + 7]);
-              *reinterpret_cast<uint4*>(stage + panel * QPANEL_BYTES + row * 128 + ((chunk ^ (row & 7)) << 4)) = val;
-            }
-          } else {
-            float4* dst = reinterpret_cast<float4*>(p.part_o + (static_cast<int64_t>(item) * BLK + row) * D + col0);
-#pragma unroll
-            for (int g = 0; g < 8; g++) dst[g] = make_float4(v[g * 4], v[g * 4 + 1], v[g * 4 + 2], v[g * 4 + 3]);
+          for (int g = 0; g < 4; g++) {
+            const int col = col0 + g * 8;
+            const int panel = col >> 6, chunk = (col & 63) >> 3;
+            uint4 val;
+            val.x = pack_bf16x2(v[g * 8 + 0], v[g * 8 + 1]);
+            val.y = pack_bf16x2(v[g * 8 + 2], v[g * 8 + 3]);
+            val.z = pack_bf16x2(v[g * 8 + 4], v[g * 8 + 5]);
+            val.w = pack_bf16x2(v[g * 8 + 6], v[g * 8 + 7]);
+            *reinterpret_cast<uint4*>(stage + panel * QPANEL_BYTES + row * 128 + ((chunk ^ (row & 7)) << 4)) = val;
           }
         }
       }
-      if (w == 0 && row < BLK) {
-        const float lse2 = mr + log2f(Lsum);
-        if (kDirectOut) {
-          if (p.lse != nullptr && qt * BLK + row < p.Nq)
-            p.lse[(static_cast<int64_t>(b) * p.H + h) * p.Nq + qt * BLK + row] = lse2 * 0.6931471805599453f;
-        } else {
-          p.part_lse2[static_cast<int64_t>(item) * BLK + row] = lse2;
-        }
-      }
-      if (kDirectOut) fence_proxy_async();
+      if (w == 0 && row < BLK && p.lse != nullptr && qt * BLK + row < p.Nq)
+        p.lse[(static_cast<int64_t>(b) * p.H + h) * p.Nq + qt * BLK + row] = (mr + log2f(Lsum)) * 0.6931471805599453f;
+      fence_proxy_async();
     }
     tc_fence_before();
     asm volatile("bar.sync 1, 256;" ::: "memory");
-    if (kDirectOut && ok && warp == 4 && lane == 0) {
+    if (ok && warp == 4 && lane == 0) {
       for (int pn = 0; pn < NPANEL; pn++)
         tma_store_4d(&tmo, smem_u32(smem + L::kQ) + pn * QPANEL_BYTES, pn * 64, qt * BLK, h, b);
       tma_store_commit();

@@ -243,7 +243,8 @@ constexpr int kSelectSmemKeys = 56 * 1024;   // 224 KB of keys at most
 
 template <bool STAGED>
 __global__ void __launch_bounds__(1024) token_select_kernel(const float* __restrict__ scores, int N, int n_protect,
-                                                            int blk, int NB, uint8_t* __restrict__ prot_tok,
+                                                            int blk, int NB, int min_tokens,
+                                                            uint8_t* __restrict__ prot_tok,
                                                             uint8_t* __restrict__ prot_blk, StatusRecord* status) {
   extern __shared__ uint32_t skeys[];
   __shared__ int bins[256];
@@ -304,9 +305,10 @@ __global__ void __launch_bounds__(1024) token_select_kernel(const float* __restr
     if (whole_bin) break;
   }
   const uint32_t T = prefix;     // the n_protect-th largest key; `want` ties at T are taken, lowest index first
-  // contiguous, 32-aligned segment per warp
-  const int seg = ((N + 31) / 32 + 31) / 32 * 32;
-  const int lo = warp * seg, hi = min(N, lo + seg);
+  // contiguous segment per warp, a whole number of blocks (blk is a multiple of 32), so that every block's
+  // count of protected tokens is known to one warp
+  const int seg = ((N + 31) / 32 + blk - 1) / blk * blk;
+  const int lo = min(N, warp * seg), hi = min(N, lo + seg);
   int eq_mine = 0;
   for (int i0 = lo; i0 < hi; i0 += 32) {
     const int i = i0 + lane;
@@ -316,6 +318,7 @@ __global__ void __launch_bounds__(1024) token_select_kernel(const float* __restr
   __syncthreads();
   int eq_seen = 0;
   for (int w2 = 0; w2 < warp; w2++) eq_seen += warp_cnt[w2];
+  int in_block = 0;     // protected tokens of the block being walked
   for (int i0 = lo; i0 < hi; i0 += 32) {
     const int i = i0 + lane;
     const bool valid = i < hi;
@@ -326,8 +329,11 @@ __global__ void __launch_bounds__(1024) token_select_kernel(const float* __restr
     const bool keep = gt || (eq && (eq_seen + __popc(eqm & ((1u << lane) - 1u))) < want);
     eq_seen += __popc(eqm);
     if (valid) ptok[i] = keep ? 1 : 0;
-    const unsigned km = __ballot_sync(0xffffffffu, keep);
-    if (km != 0u && lane == 0) pblk[i0 / blk] = 1;   // blk is a multiple of 32 and so is i0
+    in_block += __popc(__ballot_sync(0xffffffffu, keep));
+    if ((i0 + 32) % blk == 0 || i0 + 32 >= hi) {          // last 32 tokens of the block (or of the sequence)
+      if (in_block >= min_tokens && lane == 0) pblk[i0 / blk] = 1;
+      in_block = 0;
+    }
   }
 }
 
@@ -471,6 +477,8 @@ extern "C" int avsa_build_block_mask(int B, int H, int N, int d, int blk, avsa_b
   const bool given = (flags & AVSA_USE_GIVEN_BLOCK_SCORES) != 0;
   if (!given && (!tensor_ok(q, B, H) || !tensor_ok(k, B, H))) return AVSA_ERR_INVALID_ARG;
   if ((flags & (AVSA_PROTECT_ROWS | AVSA_PROTECT_COLS | AVSA_PROTECT_TOKENS)) == 0) flags |= AVSA_PROTECT_ROWS;
+  const int min_tokens = max(1, static_cast<int>((flags >> 8) & 0xffu));   // AVSA_MIN_TOKENS_PER_BLOCK(n)
+  if (min_tokens > blk) return AVSA_ERR_INVALID_ARG;
   const MaskWorkspace w = mask_ws_layout(B, H, N, d, blk);
   if (ws == nullptr || ws_bytes < w.total) return AVSA_ERR_WORKSPACE;
   cudaStream_t st = as_stream(stream);
@@ -486,10 +494,10 @@ extern "C" int avsa_build_block_mask(int B, int H, int N, int d, int blk, avsa_b
     if (cudaFuncSetAttribute(token_select_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              static_cast<int>(key_bytes)) != cudaSuccess)
       return AVSA_ERR_CUDA;
-    token_select_kernel<true><<<B, 1024, key_bytes, st>>>(scores, N, n_protect, blk, NB, ptok, pblk,
+    token_select_kernel<true><<<B, 1024, key_bytes, st>>>(scores, N, n_protect, blk, NB, min_tokens, ptok, pblk,
                                                          static_cast<StatusRecord*>(ws));
   } else {
-    token_select_kernel<false><<<B, 1024, 0, st>>>(scores, N, n_protect, blk, NB, ptok, pblk,
+    token_select_kernel<false><<<B, 1024, 0, st>>>(scores, N, n_protect, blk, NB, min_tokens, ptok, pblk,
                                                    static_cast<StatusRecord*>(ws));
   }
   if (!given) {

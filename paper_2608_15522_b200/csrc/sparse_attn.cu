@@ -14,7 +14,7 @@ static int launch_sparse_attn(int B, int H, int N, const avsa_bf16_4d& q, const 
   if (!encode_bf16_tile_map(&tv, v.ptr, B, H, N, D, v.stride_b, v.stride_h, v.stride_n, BLK)) return AVSA_ERR_CUDA;
   if (!encode_bf16_tile_map(&to, o, B, H, N, D, q.stride_b, q.stride_h, q.stride_n, BLK)) return AVSA_ERR_CUDA;
   using LF = FastSmem<BLK, D>;
-  if (cudaFuncSetAttribute(attn_fast_kernel<BLK, D, MODE_LIST>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  if (cudaFuncSetAttribute(attn_fast_kernel<BLK, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            LF::kTotal) != cudaSuccess)
     return AVSA_ERR_CUDA;
   if (cudaFuncSetAttribute(attn_redo_kernel<BLK, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal) !=
@@ -23,7 +23,7 @@ static int launch_sparse_attn(int B, int H, int N, const avsa_bf16_4d& q, const 
   dim3 grid(prm.NQT, H, B);
   // Fast kernel first; it lists the (rare) work items whose rows outgrow its fixed reference maxima, and the
   // exact-rescaling kernel behind it recomputes exactly those.
-  attn_fast_kernel<BLK, D, MODE_LIST><<<grid, kAttnThreads, LF::kTotal, st>>>(tq, tk, tv, to, prm, redo);
+  attn_fast_kernel<BLK, D><<<grid, kAttnThreads, LF::kTotal, st>>>(tq, tk, tv, to, prm, redo);
   const long long items = static_cast<long long>(prm.NQT) * H * B;
   const int redo_grid = static_cast<int>(items < 148 ? items : 148);
   attn_redo_kernel<BLK, D><<<redo_grid, kAttnThreads, L::kTotal, st>>>(tq, tk, tv, to, prm, redo);

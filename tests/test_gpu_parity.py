@@ -76,6 +76,32 @@ def test_mask_lists_bit_exact_given_oracle_scores(name, flags):
     assert np.array_equal(out["col_idx"].cpu().numpy(), idx)
 
 
+@pytest.mark.parametrize("name,min_tokens", [("tiny", 3), ("medium128", 2), ("medium128", 16), ("medium128", 128)])
+def test_mask_min_tokens_per_block_bit_exact(name, min_tokens):
+    """A block counts as protected only from `min_tokens` protected tokens on (flag bits 8-15)."""
+    w = wl.WORKLOADS[name]
+    _, _, _, s64 = _oracle_scores(w, 0)
+    q, k, _ = wl.make_self_qkv(w, 0)
+    n_protect = orc.ceil_pct(w.protect_pct, w.n_video)
+    k_keep = max(1, orc.ceil_pct(w.keep_pct, w.n_blocks))
+    bs32 = orc.block_scores(_np64(q), _np64(k), w.blk).astype(np.float32)
+    s32 = s64.astype(np.float32)
+    idx, cnt, ptok, pblk = orc.build_block_mask(bs32, s32, n_protect, k_keep, w.blk, w.n_video, True, False,
+                                                min_tokens=min_tokens)
+    any_blk = orc.protected_blocks(ptok, w.blk)
+    if name == "medium128" and min_tokens >= 16:
+        assert pblk.sum() < any_blk.sum()      # the threshold bites on these inputs
+    out = av.avsa_build_block_mask(None, None, torch.from_numpy(s32).cuda(), n_protect, k_keep, w.blk,
+                                   flags=av.AVSA_PROTECT_ROWS | av.AVSA_USE_GIVEN_BLOCK_SCORES |
+                                   av.AVSA_MIN_TOKENS_PER_BLOCK(min_tokens),
+                                   block_scores=torch.from_numpy(bs32).cuda(), shape=(w.B, w.H, w.n_video, w.d))
+    _status_ok(out["ws"])
+    assert np.array_equal(out["prot_tok"].cpu().numpy(), ptok)
+    assert np.array_equal(out["prot_blk"].cpu().numpy(), pblk)
+    assert np.array_equal(out["col_cnt"].cpu().numpy(), cnt)
+    assert np.array_equal(out["col_idx"].cpu().numpy(), idx)
+
+
 def test_mask_ties_nan_and_signed_zero_bit_exact():
     B, H, N, d, blk = 2, 2, 64 * 37 + 5, 64, 64
     NB = (N + blk - 1) // blk

@@ -177,6 +177,12 @@ def test_protected_blocks_lift():
     flags = np.zeros((1, 10), np.uint8); flags[0, [3, 9]] = 1
     assert orc.protected_blocks(flags, 4).tolist() == [[1, 0, 1]]
     assert orc.protected_blocks(np.zeros((2, 10), np.uint8), 4).tolist() == [[0, 0, 0]] * 2
+    # at least n tokens per block: block 0 holds {0,1,3}, block 1 holds {5}, the 2-token tail block holds {8,9}
+    flags = np.zeros((1, 10), np.uint8); flags[0, [0, 1, 3, 5, 8, 9]] = 1
+    assert orc.protected_blocks(flags, 4, min_tokens=1).tolist() == [[1, 1, 1]]
+    assert orc.protected_blocks(flags, 4, min_tokens=2).tolist() == [[1, 0, 1]]
+    assert orc.protected_blocks(flags, 4, min_tokens=3).tolist() == [[1, 0, 0]]
+    assert orc.protected_blocks(flags, 4, min_tokens=4).tolist() == [[0, 0, 0]]
 
 
 # ------------------------------------------------------------------------------- pooling, scores
