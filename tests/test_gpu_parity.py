@@ -275,6 +275,33 @@ def test_sparse_attention_row_maxima_growing_along_the_key_axis(step, expect_red
         assert np.all(cnt.reshape(-1)[items] > 1)
 
 
+def test_sparse_attention_is_reproducible_over_repeated_launches():
+    """Same inputs, 25 launches into fresh outputs: every result is bit-identical (the accumulation order is
+    fixed by the lists, so any difference would be a race between the pipeline's stages)."""
+    w = wl.WORKLOADS["medium128"]
+    q, k, v = (t.cuda() for t in wl.make_self_qkv(w, 9))
+    NB = w.n_blocks
+    rng = np.random.default_rng(11)
+    idx = np.full((w.B, w.H, NB, NB), -1, np.int32)
+    cnt = np.zeros((w.B, w.H, NB), np.int32)
+    for b in range(w.B):
+        for h in range(w.H):
+            for i in range(NB):
+                c = 1 + int(rng.integers(NB))
+                idx[b, h, i, :c] = np.sort(rng.choice(NB, size=c, replace=False))
+                cnt[b, h, i] = c
+    idx_d, cnt_d = torch.from_numpy(idx).cuda(), torch.from_numpy(cnt).cuda()
+    first, first_lse, ws = av.avsa_sparse_self_attn(q, k, v, idx_d, cnt_d, w.blk, want_lse=True)
+    _status_ok(ws)
+    for _ in range(24):
+        o, lse, ws = av.avsa_sparse_self_attn(q, k, v, idx_d, cnt_d, w.blk, want_lse=True)
+        assert torch.equal(o, first) and torch.equal(lse, first_lse)
+    _status_ok(ws)
+    want_o, want_l = orc.masked_attention(_np64(q), _np64(k), _np64(v), idx, cnt, w.blk)
+    _close(_np64(first), want_o, "random lists O")
+    _close(_np64(first_lse), want_l, "random lists lse")
+
+
 def test_sparse_attention_strided_bnhd_layout():
     w = wl.WORKLOADS["small128"]
     q, k, v = wl.make_self_qkv(w, 4)
