@@ -22,6 +22,8 @@ __device__ __forceinline__ uint32_t rank_key(float x) {
 // (i) block mean-pooling.  grid (NB, B*H, 2: q|k); 256 threads; each thread owns 8 channels of a
 // subset of the block's rows (16-byte loads), then the row groups are summed in a fixed order.
 // ------------------------------------------------------------------------------------------------
+constexpr unsigned kPoolTailCtas = 296;   // CTAs at the end of the pooling grid that wait for the token select
+
 template <int D>
 __global__ void __launch_bounds__(256) pool_kernel(const __nv_bfloat16* __restrict__ q, int64_t q_sb, int64_t q_sh,
                                                    int64_t q_sn, const __nv_bfloat16* __restrict__ k, int64_t k_sb,
@@ -30,6 +32,8 @@ __global__ void __launch_bounds__(256) pool_kernel(const __nv_bfloat16* __restri
   constexpr int TPR = D / 8;          // threads per row
   constexpr int RPP = 256 / TPR;      // rows per pass
   __shared__ float part[RPP][D + 4];
+  // lets the block-score grid be staged while this one drains (it waits for this grid before it reads)
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   const int nb = blockIdx.x, bh = blockIdx.y, which = blockIdx.z;
   const int b = bh / H, h = bh % H;
@@ -70,6 +74,12 @@ __global__ void __launch_bounds__(256) pool_kernel(const __nv_bfloat16* __restri
     for (int j = 0; j < RPP; j++) s += part[j][threadIdx.x];
     dst[threadIdx.x] = s / static_cast<float>(valid);
   }
+  // This grid starts while the token select (its predecessor on the stream) is still running.  The last
+  // CTAs wait for it before they retire, so that "pooling finished" implies "token select finished" for the
+  // kernels behind (which wait for their predecessor only); by then the select is long done, and no
+  // earlier CTA ever holds an SM slot waiting.
+  const unsigned lin = (blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x;
+  if (lin + kPoolTailCtas >= gridDim.x * gridDim.y * gridDim.z) asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -99,10 +109,11 @@ __global__ void __launch_bounds__(128) block_score_kernel(const float* __restric
   extern __shared__ __align__(16) float score_smem[];
   float* sq = score_smem;
   float* sk = score_smem + 64 * PITCH;
-  // Launched as an ordinary stream-ordered kernel: it starts only after both the token select and the
-  // pooling kernel (which may overlap each other) have finished.  The list kernel behind it may be
-  // scheduled early and waits for this grid.
+  // Staged behind the pooling grid (programmatic dependent launch) and waits for it here; the pooling grid
+  // in turn retires only after the token select, so the list kernel behind this one, which waits for this
+  // grid, sees the block flags too.
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   const int bh = blockIdx.z, i0 = blockIdx.y * 64, j0 = blockIdx.x * 64;
   const float* qb = qbar + static_cast<int64_t>(bh) * NB * D;
   const float* kb = kbar + static_cast<int64_t>(bh) * NB * D;
@@ -526,11 +537,23 @@ extern "C" int avsa_build_block_mask(int B, int H, int N, int d, int blk, avsa_b
       if (cudaFuncSetAttribute(block_score_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                static_cast<int>(score_smem)) != cudaSuccess)
         return AVSA_ERR_CUDA;
-      block_score_kernel<128><<<sg, 128, score_smem, st>>>(qbar, kbar, block_scores, NB, scale);
+      cfg.gridDim = sg;
+      cfg.blockDim = dim3(128, 1, 1);
+      cfg.dynamicSmemBytes = score_smem;
+      const float* qbc = qbar;
+      const float* kbc = kbar;
+      e = cudaLaunchKernelEx(&cfg, block_score_kernel<128>, qbc, kbc, block_scores, NB, scale);
+      if (e != cudaSuccess) return AVSA_ERR_CUDA;
     } else {
       e = cudaLaunchKernelEx(&cfg, pool_kernel<64>, qp, qsb, qsh, qsn, kp, ksb, ksh, ksn, qbar, kbar, H, N, blk);
       if (e != cudaSuccess) return AVSA_ERR_CUDA;
-      block_score_kernel<64><<<sg, 128, score_smem, st>>>(qbar, kbar, block_scores, NB, scale);
+      cfg.gridDim = sg;
+      cfg.blockDim = dim3(128, 1, 1);
+      cfg.dynamicSmemBytes = score_smem;
+      const float* qbc = qbar;
+      const float* kbc = kbar;
+      e = cudaLaunchKernelEx(&cfg, block_score_kernel<64>, qbc, kbc, block_scores, NB, scale);
+      if (e != cudaSuccess) return AVSA_ERR_CUDA;
     }
   }
   const int total_rows = B * H * NB;
