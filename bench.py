@@ -37,7 +37,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # summarised under profiles/ (None until a capture exists for that workload)
 NCU_TRAFFIC_BYTES = {"mid": 427.3e6,      # captured (profiles/attn_fast_kernel_mid.md)
                      "ovi": 784.0e6}      # the mid capture scaled by Q+K+V+O bytes: too large to capture under the size rule
-KERNELS_PER_STEP = 12   # cross: clear, pass 1, merge, pass 2, head sum; mask: select, pool, scores, rows; attn: clear, fast, redo
+KERNELS_PER_STEP = 12   # cross: clear, pass 1, merge, pass 2, head sum; mask: select, pool, scores, rows; attn: clear, persistent, redo
 
 
 def load_peaks():
@@ -398,7 +398,7 @@ def run_ours(args, w):
                                  "note": "Eq. 12-15 on [B,N,H*d] feature maps; reads both maps once; L2 not flushed "
                                          "between repetitions but the 406 MB exceed it"},
             "executed_tflops": achieved,
-            "roofline": {"kernel": "attn_fast_kernel<128,128> (avsa_sparse_self_attn)", "bound": "tensor",
+            "roofline": {"kernel": "attn_persist_kernel<128,128> (avsa_sparse_self_attn)", "bound": "tensor",
                          "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
                          "peak_source": f"{peak_kind} bf16_tflops (burst)", "frac_of_sustained": achieved / sustained,
                          "frac_of_nominal_2250": achieved / 2250.0,

@@ -53,6 +53,8 @@ struct AttnParams {
   const int32_t* col_idx;   // [B,H,NB,NB]
   const int32_t* col_cnt;   // [B,H,NB]
   float* lse;               // [B,H,Nq] natural log, optional
+  __nv_bfloat16* o;         // output tensor and its element strides (kernels that store rows directly)
+  int64_t o_sb, o_sh, o_sn;
   // MODE_RANGE
   float* part_o;            // [items][BLK][D] fp32
   float* part_lse2;         // [items][BLK]

@@ -17,6 +17,7 @@ struct StatusRecord {
   int item;       // work item (block index)
   int aux;        // tile index or offending value
   int redo_count; // sparse attention: work items the fast kernel left to the exact kernel in this call
+  int next_item;  // sparse attention: head of the work queue of the persistent kernel
 };
 constexpr size_t kStatusBytes = 256;   // the record, padded so that what follows stays 256-byte aligned
 
@@ -35,6 +36,7 @@ static __global__ void clear_status_kernel(StatusRecord* st) {
   st->item = 0;
   st->aux = 0;
   st->redo_count = 0;
+  st->next_item = 0;
 }
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }

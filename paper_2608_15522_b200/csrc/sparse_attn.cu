@@ -1,6 +1,6 @@
 // avsa_sparse_self_attn: block-sparse video self-attention under the protected block mask
 // (Eq. 10 / Eq. 11; Eq. 5 when every list is full).  Host side: argument checks, tensor maps, launch.
-#include "attn_fast_kernel.cuh"
+#include "attn_persist_kernel.cuh"
 
 namespace avsa {
 
@@ -23,8 +23,20 @@ static int launch_sparse_attn(int B, int H, int N, const avsa_bf16_4d& q, const 
   dim3 grid(prm.NQT, H, B);
   // Fast kernel first; it lists the (rare) work items whose rows outgrow its fixed reference maxima, and the
   // exact-rescaling kernel behind it recomputes exactly those.
-  attn_fast_kernel<BLK, D><<<grid, kAttnThreads, LF::kTotal, st>>>(tq, tk, tv, to, prm, redo);
   const long long items = static_cast<long long>(prm.NQT) * H * B;
+  // The persistent form stores rows with 32-byte accesses: it needs 32-byte-aligned rows.
+  const bool rows_aligned32 = (reinterpret_cast<uintptr_t>(o) & 31u) == 0 && q.stride_b % 16 == 0 &&
+                              q.stride_h % 16 == 0 && q.stride_n % 16 == 0;
+  if (rows_aligned32 && items <= 0x7fffffff) {
+    using LP = PersistSmem<BLK, D>;
+    if (cudaFuncSetAttribute(attn_persist_kernel<BLK, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, LP::kTotal) !=
+        cudaSuccess)
+      return AVSA_ERR_CUDA;
+    const int pgrid = static_cast<int>(items < 148 ? items : 148);
+    attn_persist_kernel<BLK, D><<<pgrid, kAttnThreads, LP::kTotal, st>>>(tq, tk, tv, prm, redo, static_cast<int>(items));
+  } else {
+    attn_fast_kernel<BLK, D><<<grid, kAttnThreads, LF::kTotal, st>>>(tq, tk, tv, to, prm, redo);
+  }
   const int redo_grid = static_cast<int>(items < 148 ? items : 148);
   attn_redo_kernel<BLK, D><<<redo_grid, kAttnThreads, L::kTotal, st>>>(tq, tk, tv, to, prm, redo);
   return cudaGetLastError() == cudaSuccess ? AVSA_OK : AVSA_ERR_CUDA;
@@ -64,6 +76,10 @@ extern "C" int avsa_sparse_self_attn(int B, int H, int N, int d, int blk, avsa_b
   prm.col_idx = col_idx;
   prm.col_cnt = col_cnt;
   prm.lse = lse;
+  prm.o = static_cast<__nv_bfloat16*>(o_bf16);
+  prm.o_sb = q.stride_b;
+  prm.o_sh = q.stride_h;
+  prm.o_sn = q.stride_n;
   prm.status = static_cast<StatusRecord*>(ws);
   prm.H = H;
   prm.Nq = N;

@@ -318,6 +318,39 @@ def test_sparse_attention_strided_bnhd_layout():
     _close(_np64(o), want, "strided O")
 
 
+def test_sparse_attention_rows_not_32_byte_aligned():
+    """Rows 272 bytes apart (d padded by 8 elements): 16-byte aligned, as the interface requires, but not
+    32-byte aligned, so the call takes the one-CTA-per-query-tile kernel with the staged TMA store instead
+    of the persistent kernel with its 32-byte row stores.  Same result either way."""
+    w = wl.WORKLOADS["medium128"]
+    q, k, v = wl.make_self_qkv(w, 12)
+    NB = w.n_blocks
+    _, _, _, s64 = _oracle_scores(w, 0)
+    n_protect = orc.ceil_pct(w.protect_pct, w.n_video)
+    k_keep = max(1, orc.ceil_pct(w.keep_pct, NB))
+    _, _, idx, cnt, _, _ = _oracle_mask(w, q, k, s64, n_protect, k_keep)
+
+    def padded(t):
+        buf = torch.zeros(t.shape[:-1] + (w.d + 8,), dtype=t.dtype, device="cuda")
+        buf[..., : w.d] = t.cuda()
+        return buf[..., : w.d]
+
+    qp, kp, vp = padded(q), padded(k), padded(v)
+    assert qp.stride(2) == w.d + 8 and qp.stride(3) == 1
+    o, lse, ws = av.avsa_sparse_self_attn(qp, kp, vp, torch.from_numpy(idx).cuda(), torch.from_numpy(cnt).cuda(), w.blk,
+                                          want_lse=True)
+    _status_ok(ws)
+    assert o.stride() == qp.stride()
+    want_o, want_l = orc.masked_attention(_np64(q), _np64(k), _np64(v), idx, cnt, w.blk)
+    _close(_np64(o), want_o, "padded rows O")
+    _close(_np64(lse), want_l, "padded rows lse")
+    # and the aligned layout gives the same numbers bit for bit (both kernels share their arithmetic)
+    o2, lse2, ws2 = av.avsa_sparse_self_attn(q.cuda(), k.cuda(), v.cuda(), torch.from_numpy(idx).cuda(),
+                                             torch.from_numpy(cnt).cuda(), w.blk, want_lse=True)
+    _status_ok(ws2)
+    assert torch.equal(o2, o.contiguous()) and torch.equal(lse2, lse)
+
+
 def test_sparse_attention_rejects_malformed_lists_without_touching_memory():
     w = wl.WORKLOADS["small128"]
     q, k, v = (t.cuda() for t in wl.make_self_qkv(w, 0))
