@@ -6,8 +6,8 @@
 // fill, and at the end the drain, the staged store and the teardown.  With one CTA per SM (shared and tensor
 // memory are both used in full) nothing overlaps that time, and a 64-tile work item lasts only about 60 us.
 // Here the roles of attn_fast_kernel loop over work items instead:
-//   * warp 0 is scheduler and K producer: it takes the next item from a global counter, checks its list, and
-//     publishes it in a two-slot ring one item ahead; its K ring simply continues into the next item's tiles,
+//   * warp 0 is scheduler and K producer: it takes the next item from a global counter (through an order
+//     array that puts the long lists first), checks its list, and publishes it in a two-slot ring one item ahead; its K ring simply continues into the next item's tiles,
 //     and Q of the next item is loaded as soon as the last Q K^T of the current one has been issued;
 //   * warp 3 (V), warp 1 (Q K^T) and warp 2 (P V) follow the published items; all ring positions and barrier
 //     phases are running counts, not per-item indices;
@@ -48,7 +48,7 @@ template <int BLK, int D>
 __global__ void __launch_bounds__(kAttnThreads, 1)
 attn_persist_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUtensorMap tmk,
                     const __grid_constant__ CUtensorMap tmv, const AttnParams p, int* __restrict__ redo_list,
-                    int n_items) {
+                    const int* __restrict__ order, int n_items) {
   using L = PersistSmem<BLK, D>;
   constexpr int NPANEL = D / 64;
   constexpr int PANEL_BYTES = BLK * 128;
@@ -164,6 +164,7 @@ attn_persist_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_consta
           pub_cnt = 0;
           break;
         }
+        id = order[id];                  // queue position -> query tile (long lists first)
         const int c = p.col_cnt[id];
         bool bad = (c < 1 || c > p.NKB);
         if (!bad) {

@@ -4,6 +4,55 @@
 
 namespace avsa {
 
+// First kernel of the call: resets the status record and writes the order in which the persistent kernel's
+// work queue hands out the query tiles -- long lists first (more than half the key blocks: the protected,
+// dense rows), short ones last, each class in index order.  With the long items at the end of the queue the
+// last CTAs to finish would leave the others idle for up to a whole dense row.
+__global__ void __launch_bounds__(1024) prep_sparse_kernel(StatusRecord* st, const int32_t* __restrict__ col_cnt,
+                                                           int n_items, int NKB, int* __restrict__ order) {
+  __shared__ int warp_tot[32];
+  __shared__ int total_heavy;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (tid == 0) {
+    st->code = 0;
+    st->where = 0;
+    st->item = 0;
+    st->aux = 0;
+    st->redo_count = 0;
+    st->next_item = 0;
+  }
+  const int chunk = (n_items + 1023) / 1024;
+  const int lo = min(n_items, tid * chunk), hi = min(n_items, lo + chunk);
+  int heavy = 0;
+  for (int i = lo; i < hi; i++) heavy += (2 * col_cnt[i] > NKB) ? 1 : 0;
+  // exclusive scan of the per-thread counts over the block
+  int incl = heavy;
+#pragma unroll
+  for (int off = 1; off < 32; off <<= 1) {
+    const int t = __shfl_up_sync(0xffffffffu, incl, off);
+    if (lane >= off) incl += t;
+  }
+  if (lane == 31) warp_tot[warp] = incl;
+  __syncthreads();
+  if (warp == 0) {
+    int w = warp_tot[lane];
+    int wi = w;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+      const int t = __shfl_up_sync(0xffffffffu, wi, off);
+      if (lane >= off) wi += t;
+    }
+    warp_tot[lane] = wi - w;
+    if (lane == 31) total_heavy = wi;
+  }
+  __syncthreads();
+  int h_pos = warp_tot[warp] + incl - heavy;          // heavy items before this thread's chunk
+  int l_pos = total_heavy + lo - h_pos;               // light items go behind all heavy ones
+  for (int i = lo; i < hi; i++) {
+    if (2 * col_cnt[i] > NKB) order[h_pos++] = i; else order[l_pos++] = i;
+  }
+}
+
 template <int BLK, int D>
 static int launch_sparse_attn(int B, int H, int N, const avsa_bf16_4d& q, const avsa_bf16_4d& k,
                               const avsa_bf16_4d& v, void* o, const AttnParams& prm, int* redo, cudaStream_t st) {
@@ -33,7 +82,8 @@ static int launch_sparse_attn(int B, int H, int N, const avsa_bf16_4d& q, const 
         cudaSuccess)
       return AVSA_ERR_CUDA;
     const int pgrid = static_cast<int>(items < 148 ? items : 148);
-    attn_persist_kernel<BLK, D><<<pgrid, kAttnThreads, LP::kTotal, st>>>(tq, tk, tv, prm, redo, static_cast<int>(items));
+    attn_persist_kernel<BLK, D><<<pgrid, kAttnThreads, LP::kTotal, st>>>(tq, tk, tv, prm, redo, redo + items,
+                                                                         static_cast<int>(items));
   } else {
     attn_fast_kernel<BLK, D><<<grid, kAttnThreads, LF::kTotal, st>>>(tq, tk, tv, to, prm, redo);
   }
@@ -57,7 +107,8 @@ extern "C" __attribute__((visibility("default"))) void avsa_debug_set_trace(long
 extern "C" size_t avsa_sparse_self_attn_workspace_bytes(int B, int H, int N, int d, int blk) {
   if (B <= 0 || H <= 0 || N <= 0 || d <= 0 || blk <= 0) return 0;
   const size_t nb = (static_cast<size_t>(N) + blk - 1) / blk;
-  return kStatusBytes + align_up(static_cast<size_t>(B) * H * nb * sizeof(int), 256);   // status + one flag per item
+  // status record, list of recomputed work items, order of the work queue
+  return kStatusBytes + align_up(static_cast<size_t>(B) * H * nb * 2 * sizeof(int), 256);
 }
 
 extern "C" int avsa_sparse_self_attn(int B, int H, int N, int d, int blk, avsa_bf16_4d q, avsa_bf16_4d k,
@@ -90,8 +141,10 @@ extern "C" int avsa_sparse_self_attn(int B, int H, int N, int d, int blk, avsa_b
 #ifdef AVSA_TRACE
   prm.trace = g_trace_buffer;
 #endif
-  clear_status_kernel<<<1, 1, 0, st>>>(prm.status);
   int* redo = reinterpret_cast<int*>(static_cast<uint8_t*>(ws) + kStatusBytes);
+  const long long n_items = static_cast<long long>(B) * H * prm.NQT;
+  if (n_items > 0x3fffffff) return AVSA_ERR_UNSUPPORTED;
+  prep_sparse_kernel<<<1, 1024, 0, st>>>(prm.status, col_cnt, static_cast<int>(n_items), prm.NKB, redo + n_items);
   if (d == 128) return launch_sparse_attn<128, 128>(B, H, N, q, k, v, o_bf16, prm, redo, st);
   return launch_sparse_attn<64, 64>(B, H, N, q, k, v, o_bf16, prm, redo, st);
 }
