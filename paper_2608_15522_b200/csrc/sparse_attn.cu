@@ -5,11 +5,15 @@
 namespace avsa {
 
 // First kernel of the call: resets the status record and writes the order in which the persistent kernel's
-// work queue hands out the query tiles -- long lists first (more than half the key blocks: the protected,
-// dense rows), short ones last, each class in index order.  With the long items at the end of the queue the
-// last CTAs to finish would leave the others idle for up to a whole dense row.
+// work queue hands out the query tiles.  Query tiles go head by head (one head's K and V stay in L2 while its
+// tiles are in flight), except for the last heads of the queue, from `tail_start` on: there the long lists
+// (more than half the key blocks: the protected, dense rows) come first and the short ones last, each class in
+// index order.  With long items at the very end of the queue, the last CTAs to finish would leave the others
+// idle for up to a whole dense row; reordering the whole queue that way would read every head's K and V twice
+// from DRAM (once per class), which is why only as many heads as fit in L2 together are reordered.
 __global__ void __launch_bounds__(1024) prep_sparse_kernel(StatusRecord* st, const int32_t* __restrict__ col_cnt,
-                                                           int n_items, int NKB, int* __restrict__ order) {
+                                                           int n_items, int tail_start, int NKB,
+                                                           int* __restrict__ order) {
   __shared__ int warp_tot[32];
   __shared__ int total_heavy;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -21,8 +25,10 @@ __global__ void __launch_bounds__(1024) prep_sparse_kernel(StatusRecord* st, con
     st->redo_count = 0;
     st->next_item = 0;
   }
-  const int chunk = (n_items + 1023) / 1024;
-  const int lo = min(n_items, tid * chunk), hi = min(n_items, lo + chunk);
+  for (int i = tid; i < tail_start; i += 1024) order[i] = i;
+  const int n_tail = n_items - tail_start;
+  const int chunk = (n_tail + 1023) / 1024;
+  const int lo = tail_start + min(n_tail, tid * chunk), hi = min(n_items, lo + chunk);
   int heavy = 0;
   for (int i = lo; i < hi; i++) heavy += (2 * col_cnt[i] > NKB) ? 1 : 0;
   // exclusive scan of the per-thread counts over the block
@@ -35,7 +41,7 @@ __global__ void __launch_bounds__(1024) prep_sparse_kernel(StatusRecord* st, con
   if (lane == 31) warp_tot[warp] = incl;
   __syncthreads();
   if (warp == 0) {
-    int w = warp_tot[lane];
+    const int w = warp_tot[lane];
     int wi = w;
 #pragma unroll
     for (int off = 1; off < 32; off <<= 1) {
@@ -46,10 +52,10 @@ __global__ void __launch_bounds__(1024) prep_sparse_kernel(StatusRecord* st, con
     if (lane == 31) total_heavy = wi;
   }
   __syncthreads();
-  int h_pos = warp_tot[warp] + incl - heavy;          // heavy items before this thread's chunk
-  int l_pos = total_heavy + lo - h_pos;               // light items go behind all heavy ones
+  int h_pos = warp_tot[warp] + incl - heavy;                      // heavy items of the tail before this thread's chunk
+  int l_pos = total_heavy + (lo - tail_start) - h_pos;            // light items go behind all heavy ones
   for (int i = lo; i < hi; i++) {
-    if (2 * col_cnt[i] > NKB) order[h_pos++] = i; else order[l_pos++] = i;
+    if (2 * col_cnt[i] > NKB) order[tail_start + h_pos++] = i; else order[tail_start + l_pos++] = i;
   }
 }
 
@@ -144,7 +150,14 @@ extern "C" int avsa_sparse_self_attn(int B, int H, int N, int d, int blk, avsa_b
   int* redo = reinterpret_cast<int*>(static_cast<uint8_t*>(ws) + kStatusBytes);
   const long long n_items = static_cast<long long>(B) * H * prm.NQT;
   if (n_items > 0x3fffffff) return AVSA_ERR_UNSUPPORTED;
-  prep_sparse_kernel<<<1, 1024, 0, st>>>(prm.status, col_cnt, static_cast<int>(n_items), prm.NKB, redo + n_items);
+  // heads whose K and V (2 x N x d bf16 each) fit into about half of the 126 MB L2 together
+  const long long kv_bytes = 4ll * N * d;
+  long long tail_heads = (64ll << 20) / kv_bytes;
+  if (tail_heads < 1) tail_heads = 1;
+  if (tail_heads > static_cast<long long>(B) * H) tail_heads = static_cast<long long>(B) * H;
+  const int tail_start = static_cast<int>((static_cast<long long>(B) * H - tail_heads) * prm.NQT);
+  prep_sparse_kernel<<<1, 1024, 0, st>>>(prm.status, col_cnt, static_cast<int>(n_items), tail_start, prm.NKB,
+                                         redo + n_items);
   if (d == 128) return launch_sparse_attn<128, 128>(B, H, N, q, k, v, o_bf16, prm, redo, st);
   return launch_sparse_attn<64, 64>(B, H, N, q, k, v, o_bf16, prm, redo, st);
 }
