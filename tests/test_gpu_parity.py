@@ -369,6 +369,42 @@ def test_sparse_attention_rejects_malformed_lists_without_touching_memory():
     assert av.avsa_read_status(ws)[0] == av.AVSA_ERR_BAD_MASK
 
 
+def test_sparse_attention_skips_only_the_malformed_item_of_a_long_queue():
+    """408 work items on 148 persistent CTAs, three of them malformed (bad count, descending entries, entry out
+    of range): the status says BAD_MASK, the malformed items' rows are left untouched, every other row is right."""
+    import dataclasses
+    w = dataclasses.replace(wl.WORKLOADS["medium128"], H=12)
+    q, k, v = wl.make_self_qkv(w, 13)
+    NB = w.n_blocks
+    rng = np.random.default_rng(14)
+    idx = np.full((w.B, w.H, NB, NB), -1, np.int32)
+    cnt = np.zeros((w.B, w.H, NB), np.int32)
+    for b in range(w.B):
+        for h in range(w.H):
+            for i in range(NB):
+                c = 1 + int(rng.integers(6))
+                idx[b, h, i, :c] = np.sort(rng.choice(NB, size=c, replace=False))
+                cnt[b, h, i] = c
+    good_idx, good_cnt = idx.copy(), cnt.copy()
+    bad_items = [(0, 3, 5), (1, 7, 0), (1, 11, 16)]
+    cnt[0, 3, 5] = NB + 1
+    idx[1, 7, 0, :2] = [4, 2]; cnt[1, 7, 0] = 2
+    idx[1, 11, 16, :1] = [NB]; cnt[1, 11, 16] = 1
+    o = torch.full((w.B, w.H, w.n_video, w.d), 7.0, dtype=torch.bfloat16, device="cuda")
+    _, _, ws = av.avsa_sparse_self_attn(q.cuda(), k.cuda(), v.cuda(), torch.from_numpy(idx).cuda(),
+                                        torch.from_numpy(cnt).cuda(), w.blk, o=o)
+    code, detail = av.avsa_read_status(ws)
+    assert code == av.AVSA_ERR_BAD_MASK
+    assert detail[1] in [(b * w.H + h) * NB + i for b, h, i in bad_items]
+    want, _ = orc.masked_attention(_np64(q), _np64(k), _np64(v), good_idx, good_cnt, w.blk)
+    got = _np64(o)
+    for b, h, i in bad_items:
+        lo, hi = i * w.blk, min((i + 1) * w.blk, w.n_video)
+        assert np.all(got[b, h, lo:hi] == 7.0)              # refused: nothing written
+        want[b, h, lo:hi] = 7.0
+    _close(got, want, "queue with malformed items")
+
+
 # ------------------------------------------------------------------------------------------- cross attention
 @pytest.mark.parametrize("name", ["tiny", "small128", "medium128"])
 def test_cross_attention_outputs_and_scores(name):
