@@ -275,6 +275,13 @@ def avsa_sparse_self_attn(q, k, v, col_idx, col_cnt, blk, softmax_scale=0.0, wan
     return o, lse, ws
 
 
+def avsa_redo_count(ws: torch.Tensor) -> int:
+    """Diagnostic: number of work items that the last attention call on this workspace (sparse self-attention,
+    cross-attention pass 1, protected rows) recomputed with the exact-rescaling kernel."""
+    torch.cuda.synchronize(ws.device)
+    return int(ws[16:20].view(torch.int32).item())
+
+
 def avsa_sparse_self_attn_redo_items(ws: torch.Tensor):
     """Diagnostic: (count, int32 array) of the work items ((b*H + h)*NB + query block) that the last
     avsa_sparse_self_attn call on this workspace recomputed with the exact-rescaling kernel."""

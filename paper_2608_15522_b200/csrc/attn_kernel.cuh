@@ -492,9 +492,9 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__
   attn_fwd_body<BLK, D, MODE>(&tmq, &tmk, &tmv, &tmo, p, blockIdx.x, blockIdx.y, blockIdx.z);
 }
 
-// Exact-rescaling pass behind attn_fast_kernel: recomputes the work items that kernel listed (normally
-// none: then every CTA of this small grid returns at once).  CTA c takes entries c, c + gridDim.x, ...
-template <int BLK, int D>
+// Exact-rescaling pass behind the fast kernels: recomputes the work items they listed (normally none: then
+// every CTA of this small grid returns at once).  CTA c takes entries c, c + gridDim.x, ...
+template <int BLK, int D, int MODE = MODE_LIST>
 __global__ void __launch_bounds__(kAttnThreads, 1)
 attn_redo_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUtensorMap tmk,
                  const __grid_constant__ CUtensorMap tmv, const __grid_constant__ CUtensorMap tmo,
@@ -504,9 +504,10 @@ attn_redo_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant_
   const int n_redo = p.status->redo_count;
   const int warp = threadIdx.x >> 5;
   for (int k = blockIdx.x; k < n_redo; k += gridDim.x) {
-    const int item = redo_list[k];                     // (b * H + h) * NQT + qt
-    const int qt = item % p.NQT, bh = item / p.NQT;
-    attn_fwd_body<BLK, D, MODE_LIST>(&tmq, &tmk, &tmv, &tmo, p, qt, bh % p.H, bh / p.H);
+    const int item = redo_list[k];                     // list mode: (b*H + h)*NQT + qt; range modes: that * n_split + split
+    const int per_bh = p.NQT * (MODE == MODE_LIST ? 1 : p.n_split);
+    const int bx = item % per_bh, bh = item / per_bh;
+    attn_fwd_body<BLK, D, MODE>(&tmq, &tmk, &tmv, &tmo, p, bx, bh % p.H, bh / p.H);
     // back to the launch state for the next item: every warp at the launch register count, barriers invalidated
     if (warp < 4) {
       asm volatile("setmaxnreg.inc.sync.aligned.u32 168;");

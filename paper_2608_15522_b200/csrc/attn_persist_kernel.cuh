@@ -44,12 +44,42 @@ __device__ __forceinline__ void st_global_v8(void* ptr, const uint32_t (&r)[8]) 
                : "memory");
 }
 
-template <int BLK, int D>
+// One work item: which query tile, which key tiles.
+struct PersistItem {
+  int qt, h, b, kb0;
+  const int32_t* list;
+};
+template <int MODE>
+__device__ __forceinline__ PersistItem decode_item(const AttnParams& p, int item) {
+  PersistItem it;
+  int rest = item;
+  it.kb0 = 0;
+  it.list = nullptr;
+  if (MODE == MODE_LIST) {
+    it.list = p.col_idx + static_cast<int64_t>(item) * p.NKB;
+  } else {
+    it.kb0 = (item % p.n_split) * p.tiles_per_split;
+    rest = item / p.n_split;
+  }
+  it.qt = rest % p.NQT;
+  const int bh = rest / p.NQT;
+  it.h = bh % p.H;
+  it.b = bh / p.H;
+  return it;
+}
+
+// MODE_LIST: work item = query tile with an explicit list of key tiles, output bf16 rows + optional LSE
+// (block-sparse self-attention; `order` maps queue position to item).  MODE_RANGE / MODE_RANGE_DIRECT: work
+// item = (query tile, split of the key axis), key tiles kb0 .. kb0+cnt-1; output normalised fp32 partials +
+// log2 LSE per split (merge_splits_kernel combines them), or bf16 rows directly when there is one split.
+template <int BLK, int D, int MODE>
 __global__ void __launch_bounds__(kAttnThreads, 1)
 attn_persist_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUtensorMap tmk,
                     const __grid_constant__ CUtensorMap tmv, const AttnParams p, int* __restrict__ redo_list,
                     const int* __restrict__ order, int n_items) {
   using L = PersistSmem<BLK, D>;
+  constexpr bool kListIn = (MODE == MODE_LIST);
+  constexpr bool kDirectOut = (MODE != MODE_RANGE);
   constexpr int NPANEL = D / 64;
   constexpr int PANEL_BYTES = BLK * 128;
   constexpr int QPANEL_BYTES = 128 * 128;
@@ -164,6 +194,12 @@ attn_persist_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_consta
           pub_cnt = 0;
           break;
         }
+        if (!kListIn) {
+          const int kb0 = (id % p.n_split) * p.tiles_per_split;
+          pub_item = id;
+          pub_cnt = min(p.NKB, kb0 + p.tiles_per_split) - kb0;
+          break;
+        }
         id = order[id];                  // queue position -> query tile (long lists first)
         const int c = p.col_cnt[id];
         bool bad = (c < 1 || c > p.NKB);
@@ -202,9 +238,8 @@ attn_persist_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_consta
     bool ok = publish(0);
     int cur_item = pub_item, cur_cnt = pub_cnt;
     while (ok && cur_item >= 0) {
-      const int qt = cur_item % p.NQT, bh = cur_item / p.NQT;
-      const int h = bh % p.H, b = bh / p.H;
-      const int32_t* list = p.col_idx + static_cast<int64_t>(cur_item) * p.NKB;
+      const PersistItem it = decode_item<MODE>(p, cur_item);
+      const int qt = it.qt, h = it.h, b = it.b;
       if (n > 0) {
         ok = wait_all(Q_EMPTY, (n - 1) & 1, kPersistQEmpty, n);     // the last Q K^T of the item before has been issued and has run
         if (!ok) break;
@@ -218,7 +253,8 @@ attn_persist_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_consta
       const int pub_at = min(cur_cnt, kStages) - 1;     // the next item is fetched once the K ring has been filled
       int nxt_item = -1, nxt_cnt = 0;
       for (int t0 = 0; t0 < cur_cnt && ok; t0 += 32) {
-        const int mine = (t0 + lane < cur_cnt) ? list[t0 + lane] : 0;
+        int mine = it.kb0 + t0 + lane;
+        if (kListIn) mine = (t0 + lane < cur_cnt) ? it.list[t0 + lane] : 0;
         const int nn = min(32, cur_cnt - t0);
         for (int j = 0; j < nn && ok; j++) {
           const int kb = __shfl_sync(FULLM, mine, j);
@@ -264,11 +300,11 @@ attn_persist_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_consta
     for (int n = 0; ok; n++) {
       int item, cnt;
       if (!get_item(n, item, cnt)) break;
-      const int bh = item / p.NQT;
-      const int h = bh % p.H, b = bh / p.H;
-      const int32_t* list = p.col_idx + static_cast<int64_t>(item) * p.NKB;
+      const PersistItem it = decode_item<MODE>(p, item);
+      const int h = it.h, b = it.b;
       for (int t0 = 0; t0 < cnt && ok; t0 += 32) {
-        const int mine = (t0 + lane < cnt) ? list[t0 + lane] : 0;
+        int mine = it.kb0 + t0 + lane;
+        if (kListIn) mine = (t0 + lane < cnt) ? it.list[t0 + lane] : 0;
         const int nn = min(32, cnt - t0);
         for (int j = 0; j < nn; j++) {
           const int kb = __shfl_sync(FULLM, mine, j);
@@ -413,10 +449,9 @@ attn_persist_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_consta
     for (int n = 0; ok; n++) {
       int item, cnt;
       if (!get_item(n, item, cnt)) break;
-      const int qt = item % p.NQT, bh = item / p.NQT;
-      const int h = bh % p.H, b = bh / p.H;
-      const int32_t* list = p.col_idx + static_cast<int64_t>(item) * p.NKB;
-      const int last_kb = list[cnt - 1];
+      const PersistItem it = decode_item<MODE>(p, item);
+      const int qt = it.qt, h = it.h, b = it.b;
+      const int last_kb = kListIn ? it.list[cnt - 1] : it.kb0 + cnt - 1;
       const int ragged_valid = (last_kb == p.NKB - 1) ? (p.Nk - last_kb * BLK) : BLK;
       float m_ref = 0.f;
       uint64_t sum2[4] = {0ull, 0ull, 0ull, 0ull};
@@ -522,20 +557,33 @@ attn_persist_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_consta
       tc_fence_before();
       mbar_arrive(BAR(O_FREE));           // the accumulator is in registers: the next item's P V may start
       const int64_t grow = static_cast<int64_t>(qt) * BLK + row;
-      if (!redo && row < BLK && grow < p.Nq) {
-        // half a row per thread, 32 bytes per store: every store fills whole sectors
-        const float inv = 1.0f / Lsum;
-        __nv_bfloat16* orow = p.o + b * p.o_sb + h * p.o_sh + grow * p.o_sn + w * HALF;
+      const float inv = 1.0f / Lsum;
+      if (kDirectOut) {
+        if (!redo && row < BLK && grow < p.Nq) {
+          // half a row per thread, 32 bytes per store: every store fills whole sectors
+          __nv_bfloat16* orow = p.o + b * p.o_sb + h * p.o_sh + grow * p.o_sn + w * HALF;
 #pragma unroll
-        for (int g = 0; g < HALF / 16; g++) {
+          for (int g = 0; g < HALF / 16; g++) {
+            uint32_t r[8];
+#pragma unroll
+            for (int i = 0; i < 8; i++)
+              r[i] = pack_bf16x2(__uint_as_float(o0[g * 16 + 2 * i]) * inv, __uint_as_float(o0[g * 16 + 2 * i + 1]) * inv);
+            st_global_v8(orow + g * 16, r);
+          }
+          if (w == 0 && p.lse != nullptr)
+            p.lse[(static_cast<int64_t>(b) * p.H + h) * p.Nq + grow] = (m_ref + log2f(Lsum)) * 0.6931471805599453f;
+        }
+      } else if (!redo && row < BLK) {
+        // normalised fp32 partial of this split + its log2 LSE, for merge_splits_kernel
+        float* prow = p.part_o + (static_cast<int64_t>(item) * BLK + row) * D + w * HALF;
+#pragma unroll
+        for (int g = 0; g < HALF / 8; g++) {
           uint32_t r[8];
 #pragma unroll
-          for (int i = 0; i < 8; i++)
-            r[i] = pack_bf16x2(__uint_as_float(o0[g * 16 + 2 * i]) * inv, __uint_as_float(o0[g * 16 + 2 * i + 1]) * inv);
-          st_global_v8(orow + g * 16, r);
+          for (int i = 0; i < 8; i++) r[i] = __float_as_uint(__uint_as_float(o0[g * 8 + i]) * inv);
+          st_global_v8(prow + g * 8, r);
         }
-        if (w == 0 && p.lse != nullptr)
-          p.lse[(static_cast<int64_t>(b) * p.H + h) * p.Nq + grow] = (m_ref + log2f(Lsum)) * 0.6931471805599453f;
+        if (w == 0) p.part_lse2[static_cast<int64_t>(item) * BLK + row] = m_ref + log2f(Lsum);
       }
       item_done(n);
     }

@@ -3,7 +3,7 @@
 //   pass 1  flash attention, key axis split across CTAs -> partial (O, LSE) -> merge -> O, row LSE
 //   pass 2  for every key tile: S^T = K Q^T on the tensor cores, p = exp2(S^T c - lse_j), summed over
 //           the queries -> per-head column sums -> fixed-order head sum with the beta/gamma blend
-#include "attn_kernel.cuh"
+#include "attn_persist_kernel.cuh"
 
 namespace avsa {
 
@@ -415,7 +415,7 @@ struct CrossPlan {
   int NKT, NCH, W, n_range, tpr;             // pass 2 (key tiles of 128)
   bool reverse;                              // pass 2 with the keys resident (Nq > 512, Nk <= 512)
   int NQC, rev_ranges, rev_cpr, rev_slots;   // query chunks of 128, CTAs per (b,h), chunks per CTA, partial slots
-  size_t off_part_o, off_part_lse, off_lse, off_lse2, off_partial, total;
+  size_t off_part_o, off_part_lse, off_lse, off_lse2, off_partial, off_redo, total;
 };
 
 static CrossPlan make_cross_plan(int B, int H, int Nq, int Nk, int d) {
@@ -456,6 +456,7 @@ static CrossPlan make_cross_plan(int B, int H, int Nq, int Nk, int d) {
   c.off_lse2 = off; off += c.reverse ? align_up(static_cast<size_t>(B) * H * c.NQC * 128 * sizeof(float), 256) : 0;
   const size_t slots = c.reverse ? static_cast<size_t>(c.rev_slots) : static_cast<size_t>(c.NCH);
   c.off_partial = off; off += align_up(slots * B * H * Nk * sizeof(float), 256);
+  c.off_redo = off; off += align_up(items * sizeof(int), 256);
   c.total = off;
   return c;
 }
@@ -477,9 +478,7 @@ static int run_cross(int B, int H, int Nq, int Nk, const avsa_bf16_4d& q, const 
     if (!encode_bf16_tile_map(&tq, q.ptr, B, H, Nq, D, q.stride_b, q.stride_h, q.stride_n, BLK)) return AVSA_ERR_CUDA;
     if (!encode_bf16_tile_map(&tk, k.ptr, B, H, Nk, D, k.stride_b, k.stride_h, k.stride_n, BLK)) return AVSA_ERR_CUDA;
     if (!encode_bf16_tile_map(&tv, v.ptr, B, H, Nk, D, v.stride_b, v.stride_h, v.stride_n, BLK)) return AVSA_ERR_CUDA;
-    if (cudaFuncSetAttribute(attn_fwd_kernel<BLK, D, MODE_RANGE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             L::kTotal) != cudaSuccess)
-      return AVSA_ERR_CUDA;
+    using LP = PersistSmem<BLK, D>;
     AttnParams prm = {};
     prm.part_o = part_o;
     prm.part_lse2 = part_lse;
@@ -492,7 +491,11 @@ static int run_cross(int B, int H, int Nq, int Nk, const avsa_bf16_4d& q, const 
     prm.Nk = Nk;
     prm.NKB = c.NKB;
     prm.scale_log2 = scale * 1.4426950408889634f;
-    dim3 grid(c.NQT * c.n_split, H, B);
+    // Pass 1 runs on the persistent fast kernel (one CTA per SM over the (query tile, key split) items), with the
+    // exact-rescaling kernel behind it for the items whose rows outgrow their first-tile reference.
+    int* redo = reinterpret_cast<int*>(ws + c.off_redo);
+    const long long items = static_cast<long long>(B) * H * c.NQT * c.n_split;
+    const int pgrid = static_cast<int>(items < 148 ? items : 148);
     if (c.n_split == 1 && o != nullptr) {
       // the whole key axis fits one work item (few keys): write O and the LSE directly, no partials to merge
       CUtensorMap to;
@@ -501,9 +504,36 @@ static int run_cross(int B, int H, int Nq, int Nk, const avsa_bf16_4d& q, const 
                                L::kTotal) != cudaSuccess)
         return AVSA_ERR_CUDA;
       prm.lse = lse;
-      attn_fwd_kernel<BLK, D, MODE_RANGE_DIRECT><<<grid, kAttnThreads, L::kTotal, st>>>(tq, tk, tv, to, prm);
+      prm.o = static_cast<__nv_bfloat16*>(o);
+      prm.o_sb = q.stride_b;
+      prm.o_sh = q.stride_h;
+      prm.o_sn = q.stride_n;
+      const bool rows_aligned32 = (reinterpret_cast<uintptr_t>(o) & 31u) == 0 && q.stride_b % 16 == 0 &&
+                                  q.stride_h % 16 == 0 && q.stride_n % 16 == 0;
+      if (rows_aligned32) {
+        if (cudaFuncSetAttribute(attn_persist_kernel<BLK, D, MODE_RANGE_DIRECT>,
+                                 cudaFuncAttributeMaxDynamicSharedMemorySize, LP::kTotal) != cudaSuccess)
+          return AVSA_ERR_CUDA;
+        if (cudaFuncSetAttribute(attn_redo_kernel<BLK, D, MODE_RANGE_DIRECT>,
+                                 cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal) != cudaSuccess)
+          return AVSA_ERR_CUDA;
+        attn_persist_kernel<BLK, D, MODE_RANGE_DIRECT><<<pgrid, kAttnThreads, LP::kTotal, st>>>(
+            tq, tk, tv, prm, redo, nullptr, static_cast<int>(items));
+        attn_redo_kernel<BLK, D, MODE_RANGE_DIRECT><<<pgrid, kAttnThreads, L::kTotal, st>>>(tq, tk, tv, to, prm, redo);
+      } else {
+        dim3 grid(c.NQT * c.n_split, H, B);
+        attn_fwd_kernel<BLK, D, MODE_RANGE_DIRECT><<<grid, kAttnThreads, L::kTotal, st>>>(tq, tk, tv, to, prm);
+      }
     } else {
-      attn_fwd_kernel<BLK, D, MODE_RANGE><<<grid, kAttnThreads, L::kTotal, st>>>(tq, tk, tv, tq, prm);
+      if (cudaFuncSetAttribute(attn_persist_kernel<BLK, D, MODE_RANGE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               LP::kTotal) != cudaSuccess)
+        return AVSA_ERR_CUDA;
+      if (cudaFuncSetAttribute(attn_redo_kernel<BLK, D, MODE_RANGE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               L::kTotal) != cudaSuccess)
+        return AVSA_ERR_CUDA;
+      attn_persist_kernel<BLK, D, MODE_RANGE><<<pgrid, kAttnThreads, LP::kTotal, st>>>(tq, tk, tv, prm, redo, nullptr,
+                                                                                       static_cast<int>(items));
+      attn_redo_kernel<BLK, D, MODE_RANGE><<<pgrid, kAttnThreads, L::kTotal, st>>>(tq, tk, tv, tq, prm, redo);
       const int total_rows = B * H * Nq;
       constexpr int RPB = 128 / (D / 4);
       merge_splits_kernel<BLK, D><<<(total_rows + RPB - 1) / RPB, 128, 0, st>>>(

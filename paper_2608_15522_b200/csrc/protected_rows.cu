@@ -3,7 +3,7 @@
 // paper's implementation notes call it dense-row recomputation.  The protected query rows are
 // gathered into compact tiles, run densely through the attention tile kernel with the key axis split
 // across CTAs, and the merged rows overwrite the sparse result in place.
-#include "attn_kernel.cuh"
+#include "attn_persist_kernel.cuh"
 
 namespace avsa {
 
@@ -23,6 +23,8 @@ __global__ void __launch_bounds__(1024) compact_rows_kernel(const uint8_t* __res
     status->where = 0;
     status->item = 0;
     status->aux = 0;
+    status->redo_count = 0;
+    status->next_item = 0;
   }
   for (int i = tid; i < n_pad; i += 1024) out[i] = -1;
   const int seg = ((N + 31) / 32 + 31) / 32 * 32;
@@ -70,7 +72,7 @@ __global__ void __launch_bounds__(256) gather_rows_kernel(const __nv_bfloat16* _
 
 struct ProtPlan {
   int n_pad, NQT, NKB, n_split, tps;
-  size_t off_rows, off_qp, off_part_o, off_part_lse, total;
+  size_t off_rows, off_qp, off_part_o, off_part_lse, off_redo, total;
 };
 
 static ProtPlan make_prot_plan(int B, int H, int N, int d, int blk, int n_protect) {
@@ -91,6 +93,7 @@ static ProtPlan make_prot_plan(int B, int H, int N, int d, int blk, int n_protec
   c.off_qp = off; off += align_up(static_cast<size_t>(B) * H * c.n_pad * d * 2, 256);
   c.off_part_o = off; off += align_up(items * blk * d * sizeof(float), 256);
   c.off_part_lse = off; off += align_up(items * blk * sizeof(float), 256);
+  c.off_redo = off; off += align_up(items * sizeof(int), 256);
   c.total = off;
   return c;
 }
@@ -115,7 +118,11 @@ static int run_protected(int B, int H, int N, int n_protect, const avsa_bf16_4d&
     return AVSA_ERR_CUDA;
   if (!encode_bf16_tile_map(&tk, k.ptr, B, H, N, D, k.stride_b, k.stride_h, k.stride_n, BLK)) return AVSA_ERR_CUDA;
   if (!encode_bf16_tile_map(&tv, v.ptr, B, H, N, D, v.stride_b, v.stride_h, v.stride_n, BLK)) return AVSA_ERR_CUDA;
-  if (cudaFuncSetAttribute(attn_fwd_kernel<BLK, D, MODE_RANGE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  using LP = PersistSmem<BLK, D>;
+  if (cudaFuncSetAttribute(attn_persist_kernel<BLK, D, MODE_RANGE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           LP::kTotal) != cudaSuccess)
+    return AVSA_ERR_CUDA;
+  if (cudaFuncSetAttribute(attn_redo_kernel<BLK, D, MODE_RANGE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            L::kTotal) != cudaSuccess)
     return AVSA_ERR_CUDA;
   AttnParams prm = {};
@@ -130,8 +137,13 @@ static int run_protected(int B, int H, int N, int n_protect, const avsa_bf16_4d&
   prm.Nk = N;
   prm.NKB = c.NKB;
   prm.scale_log2 = scale * 1.4426950408889634f;
-  attn_fwd_kernel<BLK, D, MODE_RANGE><<<dim3(c.NQT * c.n_split, H, B), kAttnThreads, L::kTotal, st>>>(tq, tk, tv, tq,
-                                                                                                    prm);
+  // persistent fast kernel over the (row tile, key split) items, then the exact kernel for what it handed over
+  int* redo = reinterpret_cast<int*>(ws + c.off_redo);
+  const long long items = static_cast<long long>(B) * H * c.NQT * c.n_split;
+  const int grid = static_cast<int>(items < 148 ? items : 148);
+  attn_persist_kernel<BLK, D, MODE_RANGE><<<grid, kAttnThreads, LP::kTotal, st>>>(tq, tk, tv, prm, redo, nullptr,
+                                                                                  static_cast<int>(items));
+  attn_redo_kernel<BLK, D, MODE_RANGE><<<grid, kAttnThreads, L::kTotal, st>>>(tq, tk, tv, tq, prm, redo);
   const int total_rows = B * H * c.n_pad;
   constexpr int MRPB = 128 / (D / 4);
   merge_splits_kernel<BLK, D><<<(total_rows + MRPB - 1) / MRPB, 128, 0, st>>>(

@@ -84,11 +84,11 @@ static int launch_sparse_attn(int B, int H, int N, const avsa_bf16_4d& q, const 
                               q.stride_h % 16 == 0 && q.stride_n % 16 == 0;
   if (rows_aligned32 && items <= 0x7fffffff) {
     using LP = PersistSmem<BLK, D>;
-    if (cudaFuncSetAttribute(attn_persist_kernel<BLK, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, LP::kTotal) !=
+    if (cudaFuncSetAttribute(attn_persist_kernel<BLK, D, MODE_LIST>, cudaFuncAttributeMaxDynamicSharedMemorySize, LP::kTotal) !=
         cudaSuccess)
       return AVSA_ERR_CUDA;
     const int pgrid = static_cast<int>(items < 148 ? items : 148);
-    attn_persist_kernel<BLK, D><<<pgrid, kAttnThreads, LP::kTotal, st>>>(tq, tk, tv, prm, redo, redo + items,
+    attn_persist_kernel<BLK, D, MODE_LIST><<<pgrid, kAttnThreads, LP::kTotal, st>>>(tq, tk, tv, prm, redo, redo + items,
                                                                          static_cast<int>(items));
   } else {
     attn_fast_kernel<BLK, D><<<grid, kAttnThreads, LF::kTotal, st>>>(tq, tk, tv, to, prm, redo);

@@ -464,6 +464,29 @@ def test_cross_attention_reverse_direction(name):
     assert torch.equal(s, s2)                                              # fixed summation order
 
 
+@pytest.mark.parametrize("reverse", [False, True])
+def test_cross_attention_row_maxima_growing_along_the_key_axis(reverse):
+    """Pass 1 runs on the fast kernel too (key axis split across work items, or one item per query tile in the
+    reverse direction): with logits that grow steeply from key block to key block its rows outgrow their
+    first-tile reference and the exact-rescaling kernel must take the items over."""
+    import dataclasses
+    w = dataclasses.replace(wl.WORKLOADS["medium128"], H=12)      # forward: 24 query tiles -> key splits of 3 tiles
+    qa, kc, vc = wl.make_cross_qkv(w, 3)
+    if reverse:
+        qa, kc, vc = kc, torch.cat([qa, qa, qa], dim=2), torch.cat([qa, qa, qa], dim=2).flip(2)   # 2070 queries, 216 keys
+    u = 1.0 / np.sqrt(w.d)
+    qa = (qa.float() + 8.0 * u).to(torch.bfloat16)
+    nk = kc.shape[2]
+    ramp = torch.arange(nk, dtype=torch.float32).div(w.blk, rounding_mode="floor") * (80.0 if reverse else 48.0)
+    kc = (kc.float() + (ramp * u).view(1, 1, -1, 1)).to(torch.bfloat16)
+    o, lse, _, ws = av.avsa_cross_attn_scores(qa.cuda(), kc.cuda(), vc.cuda(), want_scores=False)
+    _status_ok(ws)
+    assert av.avsa_redo_count(ws) > 0
+    want_o, want_lse, _ = orc.cross_attention(_np64(qa), _np64(kc), _np64(vc))
+    _close(_np64(o), want_o, "growing maxima cross O")
+    _close(_np64(lse), want_lse, "growing maxima cross lse")
+
+
 def test_cross_attention_scores_need_one_short_axis():
     """Neither the queries nor the keys of a head fit on chip: the score pass is refused on the host."""
     q = torch.zeros((1, 1, 1024, 128), dtype=torch.bfloat16, device="cuda")
