@@ -52,6 +52,15 @@ bool device_is_sm100() {
   return major == 10;
 }
 
+// Grid size of the persistent kernels: one CTA per SM of the current device, at most one per work item.
+int persistent_grid(long long items) {
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1)
+    sms = 148;
+  return static_cast<int>(items < sms ? items : sms);
+}
+
 }  // namespace avsa
 
 extern "C" {

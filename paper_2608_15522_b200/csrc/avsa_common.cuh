@@ -62,6 +62,9 @@ bool encode_bf16_tile_map(CUtensorMap* map, const void* ptr, int B, int H, int N
 // True when the current device is compute capability 10.x.
 bool device_is_sm100();
 
+// Grid size of the persistent kernels: one CTA per SM of the current device, at most one per work item.
+int persistent_grid(long long items);
+
 inline cudaStream_t as_stream(void* s) { return reinterpret_cast<cudaStream_t>(s); }
 
 }  // namespace avsa

@@ -495,7 +495,7 @@ static int run_cross(int B, int H, int Nq, int Nk, const avsa_bf16_4d& q, const 
     // exact-rescaling kernel behind it for the items whose rows outgrow their first-tile reference.
     int* redo = reinterpret_cast<int*>(ws + c.off_redo);
     const long long items = static_cast<long long>(B) * H * c.NQT * c.n_split;
-    const int pgrid = static_cast<int>(items < 148 ? items : 148);
+    const int pgrid = persistent_grid(items);
     if (c.n_split == 1 && o != nullptr) {
       // the whole key axis fits one work item (few keys): write O and the LSE directly, no partials to merge
       CUtensorMap to;

@@ -76,8 +76,8 @@ static int launch_sparse_attn(int B, int H, int N, const avsa_bf16_4d& q, const 
       cudaSuccess)
     return AVSA_ERR_CUDA;
   dim3 grid(prm.NQT, H, B);
-  // Fast kernel first; it lists the (rare) work items whose rows outgrow its fixed reference maxima, and the
-  // exact-rescaling kernel behind it recomputes exactly those.
+  // The fast kernel (persistent form when the rows allow it) first; it lists the (rare) work items whose rows
+  // outgrow its fixed reference maxima, and the exact-rescaling kernel behind it recomputes exactly those.
   const long long items = static_cast<long long>(prm.NQT) * H * B;
   // The persistent form stores rows with 32-byte accesses: it needs 32-byte-aligned rows.
   const bool rows_aligned32 = (reinterpret_cast<uintptr_t>(o) & 31u) == 0 && q.stride_b % 16 == 0 &&
@@ -87,13 +87,13 @@ static int launch_sparse_attn(int B, int H, int N, const avsa_bf16_4d& q, const 
     if (cudaFuncSetAttribute(attn_persist_kernel<BLK, D, MODE_LIST>, cudaFuncAttributeMaxDynamicSharedMemorySize, LP::kTotal) !=
         cudaSuccess)
       return AVSA_ERR_CUDA;
-    const int pgrid = static_cast<int>(items < 148 ? items : 148);
+    const int pgrid = persistent_grid(items);
     attn_persist_kernel<BLK, D, MODE_LIST><<<pgrid, kAttnThreads, LP::kTotal, st>>>(tq, tk, tv, prm, redo, redo + items,
                                                                          static_cast<int>(items));
   } else {
     attn_fast_kernel<BLK, D><<<grid, kAttnThreads, LF::kTotal, st>>>(tq, tk, tv, to, prm, redo);
   }
-  const int redo_grid = static_cast<int>(items < 148 ? items : 148);
+  const int redo_grid = persistent_grid(items);
   attn_redo_kernel<BLK, D><<<redo_grid, kAttnThreads, L::kTotal, st>>>(tq, tk, tv, to, prm, redo);
   return cudaGetLastError() == cudaSuccess ? AVSA_OK : AVSA_ERR_CUDA;
 }
