@@ -318,6 +318,34 @@ def test_sparse_attention_strided_bnhd_layout():
     _close(_np64(o), want, "strided O")
 
 
+@pytest.mark.parametrize("seed", range(8))
+def test_sparse_attention_random_shapes_and_lists(seed):
+    """Seeded random shapes (batch, heads, length incl. ragged tails and lengths below one block, both tile
+    sizes) with random ascending lists of random length, against the oracle."""
+    rng = np.random.default_rng(100 + seed)
+    d = int(rng.choice([64, 128]))
+    blk = d
+    B, H = int(rng.integers(1, 4)), int(rng.integers(1, 6))
+    N = int(rng.integers(1, 9 * blk))
+    NB = (N + blk - 1) // blk
+    g = torch.Generator().manual_seed(200 + seed)
+    q, k, v = (torch.randn(B, H, N, d, generator=g).to(torch.bfloat16) for _ in range(3))
+    idx = np.full((B, H, NB, NB), -1, np.int32)
+    cnt = np.zeros((B, H, NB), np.int32)
+    for b in range(B):
+        for h in range(H):
+            for i in range(NB):
+                c = 1 + int(rng.integers(NB))
+                idx[b, h, i, :c] = np.sort(rng.choice(NB, size=c, replace=False))
+                cnt[b, h, i] = c
+    o, lse, ws = av.avsa_sparse_self_attn(q.cuda(), k.cuda(), v.cuda(), torch.from_numpy(idx).cuda(),
+                                          torch.from_numpy(cnt).cuda(), blk, want_lse=True)
+    _status_ok(ws)
+    want_o, want_l = orc.masked_attention(_np64(q), _np64(k), _np64(v), idx, cnt, blk)
+    _close(_np64(o), want_o, f"random shape B{B} H{H} N{N} d{d} O")
+    _close(_np64(lse), want_l, f"random shape B{B} H{H} N{N} d{d} lse")
+
+
 def test_sparse_attention_rows_not_32_byte_aligned():
     """Rows 272 bytes apart (d padded by 8 elements): 16-byte aligned, as the interface requires, but not
     32-byte aligned, so the call takes the one-CTA-per-query-tile kernel with the staged TMA store instead
