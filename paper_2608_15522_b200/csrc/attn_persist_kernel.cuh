@@ -21,15 +21,19 @@
 
 namespace avsa {
 
+// K stages, V stages, Q buffers.  Measured on the Ovi-class layer and on one-tile lists: (3,3,1), (3,2,2), (2,3,2),
+// (4,2,1) and (2,4,1) are all within noise of each other, so the simplest split of the 226 KB stays.
+constexpr int kPKS = 3, kPVS = 3, kPQB = 1;
+
 template <int BLK, int D>
 struct PersistSmem {
   static constexpr int kTileBytes = BLK * D * 2;
   static constexpr int kQBytes = 128 * D * 2;
   static constexpr int kQ = 0;
-  static constexpr int kK = kQBytes;
-  static constexpr int kV = kK + kStages * kTileBytes;
-  static constexpr int kBars = kV + kStages * kTileBytes;
-  static constexpr int kNumBars = 2 + 4 * kStages + 2 + 2 + 4 + 2 + 2 + 1 + 4 + 2 + 2;
+  static constexpr int kK = kPQB * kQBytes;
+  static constexpr int kV = kK + kPKS * kTileBytes;
+  static constexpr int kBars = kV + kPVS * kTileBytes;
+  static constexpr int kNumBars = 2 * kPQB + 2 * kPKS + 2 * kPVS + 21;
   static constexpr int kStats = kBars + kNumBars * 8;          // float mref[128], lsum[2][128]
   static constexpr int kItems = kStats + 3 * 128 * 4;          // int {item, cnt}[2], redo flag
   static constexpr int kMisc = kItems + 32;                    // tmem base, stop flag
@@ -93,8 +97,8 @@ attn_persist_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_consta
   }
   const uint32_t bar0 = smem_u32(smem + L::kBars);
   auto BAR = [&](int i) { return bar0 + static_cast<uint32_t>(i) * 8u; };
-  constexpr int Q_FULL = 0, Q_EMPTY = 1, K_FULL = 2, K_EMPTY = 2 + kStages, V_FULL = 2 + 2 * kStages,
-                V_EMPTY = 2 + 3 * kStages, S_FULL = 2 + 4 * kStages /* + group */, S_FREE = S_FULL + 2,
+  constexpr int Q_FULL = 0, Q_EMPTY = kPQB, K_FULL = 2 * kPQB, K_EMPTY = K_FULL + kPKS, V_FULL = K_EMPTY + kPKS,
+                V_EMPTY = V_FULL + kPVS, S_FULL = V_EMPTY + kPVS /* + group */, S_FREE = S_FULL + 2,
                 P_FULL = S_FREE + 2 /* + 2*group + half */, P_FREE = P_FULL + 4, O_FULL = P_FREE + 2,
                 O_FREE = O_FULL + 1, MREF = O_FREE + 1, ITEM_FULL = MREF + 1 /* + slot */, ITEM_EMPTY = ITEM_FULL + 2,
                 QK_DRAIN = ITEM_EMPTY + 2, PV_DRAIN = QK_DRAIN + 1, LSUM_A = PV_DRAIN + 1, LSUM_B = LSUM_A + 1;
@@ -108,11 +112,15 @@ attn_persist_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_consta
   volatile uint32_t* misc = reinterpret_cast<volatile uint32_t*>(smem + L::kMisc);   // [0] tmem base, [1] stop
 
   if (tid == 0) {
-    mbar_init(BAR(Q_FULL), 1);
-    mbar_init(BAR(Q_EMPTY), 1);
-    for (int s = 0; s < kStages; s++) {
+    for (int s = 0; s < kPQB; s++) {
+      mbar_init(BAR(Q_FULL + s), 1);
+      mbar_init(BAR(Q_EMPTY + s), 1);
+    }
+    for (int s = 0; s < kPKS; s++) {
       mbar_init(BAR(K_FULL + s), 1);
       mbar_init(BAR(K_EMPTY + s), 1);
+    }
+    for (int s = 0; s < kPVS; s++) {
       mbar_init(BAR(V_FULL + s), 1);
       mbar_init(BAR(V_EMPTY + s), 1);
     }
@@ -240,17 +248,20 @@ attn_persist_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_consta
     while (ok && cur_item >= 0) {
       const PersistItem it = decode_item<MODE>(p, cur_item);
       const int qt = it.qt, h = it.h, b = it.b;
-      if (n > 0) {
-        ok = wait_all(Q_EMPTY, (n - 1) & 1, kPersistQEmpty, n);     // the last Q K^T of the item before has been issued and has run
+      const int qb = n % kPQB;
+      if (n >= kPQB) {
+        // the last Q K^T of the item that used this Q buffer has run
+        ok = wait_all(Q_EMPTY + qb, ((n / kPQB) - 1) & 1, kPersistQEmpty, n);
         if (!ok) break;
       }
       if (lane == 0) {
-        mbar_expect_tx(BAR(Q_FULL), BLK * D * 2);
+        mbar_expect_tx(BAR(Q_FULL + qb), BLK * D * 2);
         for (int pn = 0; pn < NPANEL; pn++)
-          tma_load_4d(smem_u32(smem + L::kQ) + pn * QPANEL_BYTES, &tmq, BAR(Q_FULL), pn * 64, qt * BLK, h, b);
+          tma_load_4d(smem_u32(smem + L::kQ) + qb * L::kQBytes + pn * QPANEL_BYTES, &tmq, BAR(Q_FULL + qb), pn * 64,
+                      qt * BLK, h, b);
         q_loads++;
       }
-      const int pub_at = min(cur_cnt, kStages) - 1;     // the next item is fetched once the K ring has been filled
+      const int pub_at = min(cur_cnt, kPKS) - 1;     // the next item is fetched once the K ring has been filled
       int nxt_item = -1, nxt_cnt = 0;
       for (int t0 = 0; t0 < cur_cnt && ok; t0 += 32) {
         int mine = it.kb0 + t0 + lane;
@@ -259,10 +270,10 @@ attn_persist_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_consta
         for (int j = 0; j < nn && ok; j++) {
           const int kb = __shfl_sync(FULLM, mine, j);
           const int t = t0 + j;
-          const int s = kc % kStages;
+          const int s = kc % kPKS;
           int good = 1;
           if (lane == 0) {
-            if (kc >= kStages) good = wait_or_stop(K_EMPTY + s, ((kc / kStages) - 1) & 1, kWhereKEmpty, t) ? 1 : 0;
+            if (kc >= kPKS) good = wait_or_stop(K_EMPTY + s, ((kc / kPKS) - 1) & 1, kWhereKEmpty, t) ? 1 : 0;
             if (good) {
               mbar_expect_tx(BAR(K_FULL + s), L::kTileBytes);
               for (int pn = 0; pn < NPANEL; pn++)
@@ -289,8 +300,8 @@ attn_persist_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_consta
     }
     if (lane == 0 && misc[1] != 0u) {
       // stopped: loads still in flight must land before this CTA's shared memory is given away
-      if (q_loads > 0) mbar_wait(BAR(Q_FULL), (q_loads - 1) & 1);
-      for (int c = max(0, kc - kStages); c < kc; c++) mbar_wait(BAR(K_FULL + c % kStages), (c / kStages) & 1);
+      for (int c = max(0, q_loads - kPQB); c < q_loads; c++) mbar_wait(BAR(Q_FULL + c % kPQB), (c / kPQB) & 1);
+      for (int c = max(0, kc - kPKS); c < kc; c++) mbar_wait(BAR(K_FULL + c % kPKS), (c / kPKS) & 1);
     }
   } else if (warp == 3) {
     // ------------------------------------------------------------------ TMA producer of V
@@ -308,10 +319,10 @@ attn_persist_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_consta
         const int nn = min(32, cnt - t0);
         for (int j = 0; j < nn; j++) {
           const int kb = __shfl_sync(FULLM, mine, j);
-          const int s = vc % kStages;
+          const int s = vc % kPVS;
           int good = 1;
           if (lane == 0) {
-            if (vc >= kStages) good = wait_or_stop(V_EMPTY + s, ((vc / kStages) - 1) & 1, kWhereVEmpty, t0 + j) ? 1 : 0;
+            if (vc >= kPVS) good = wait_or_stop(V_EMPTY + s, ((vc / kPVS) - 1) & 1, kWhereVEmpty, t0 + j) ? 1 : 0;
             if (good) {
               mbar_expect_tx(BAR(V_FULL + s), L::kTileBytes);
               for (int pn = 0; pn < NPANEL; pn++)
@@ -330,7 +341,7 @@ attn_persist_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_consta
       if (ok) item_done(n);
     }
     if (lane == 0 && misc[1] != 0u)
-      for (int c = max(0, vc - kStages); c < vc; c++) mbar_wait(BAR(V_FULL + c % kStages), (c / kStages) & 1);
+      for (int c = max(0, vc - kPVS); c < vc; c++) mbar_wait(BAR(V_FULL + c % kPVS), (c / kPVS) & 1);
   } else if (warp == 1) {
     // ------------------------------------------------------------------ Q K^T issuer
     asm volatile("setmaxnreg.dec.sync.aligned.u32 64;");
@@ -339,7 +350,7 @@ attn_persist_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_consta
     constexpr uint32_t idesc_qk = make_idesc_bf16(128, BLK, 0, 0);
     const uint32_t tmem_u = __shfl_sync(FULLM, tmem, 0);
     auto desc64 = [](uint32_t lo) { return (static_cast<uint64_t>(desc_hi) << 32) | lo; };
-    const uint32_t q_lo = ((smem_u32(smem + L::kQ) & 0x3FFFFu) >> 4) | (1u << 16);
+    const uint32_t q_lo0 = ((smem_u32(smem + L::kQ) & 0x3FFFFu) >> 4) | (1u << 16);
     const uint32_t k_lo0 = ((smem_u32(smem + L::kK) & 0x3FFFFu) >> 4) | (1u << 16);
     int kc = 0;                 // K tiles consumed so far
     int used[2] = {0, 0};       // S tiles written so far into each group's buffer
@@ -347,10 +358,12 @@ attn_persist_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_consta
     for (int n = 0; ok; n++) {
       int item, cnt;
       if (!get_item(n, item, cnt)) break;
-      ok = wait_all(Q_FULL, n & 1, kWhereQFull, n);
+      const int qb = n % kPQB;
+      const uint32_t q_lo = q_lo0 + qb * (L::kQBytes >> 4);
+      ok = wait_all(Q_FULL + qb, (n / kPQB) & 1, kWhereQFull, n);
       for (int t = 0; t < cnt && ok; t++) {
-        const int j = t & 1, sk = kc % kStages;
-        ok = wait_all(K_FULL + sk, (kc / kStages) & 1, kWhereKFull, t);
+        const int j = t & 1, sk = kc % kPKS;
+        ok = wait_all(K_FULL + sk, (kc / kPKS) & 1, kWhereKFull, t);
         if (!ok) break;
         if (used[j] > 0) {
           ok = wait_all(S_FREE + j, (used[j] - 1) & 1, kFastSFree, t);     // the group has taken its last tile out
@@ -368,7 +381,7 @@ attn_persist_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_consta
           }
           umma_commit(BAR(S_FULL + j));
           umma_commit(BAR(K_EMPTY + sk));
-          if (t == cnt - 1) umma_commit(BAR(Q_EMPTY));     // Q may be replaced once this product has run
+          if (t == cnt - 1) umma_commit(BAR(Q_EMPTY + qb));     // Q may be replaced once this product has run
         }
         __syncwarp();
         used[j]++;
@@ -404,8 +417,8 @@ attn_persist_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_consta
       int item, cnt;
       if (!get_item(n, item, cnt)) break;
       for (int t = 0; t < cnt && ok; t++) {
-        const int j = t & 1, sv = vc % kStages;
-        ok = wait_all(V_FULL + sv, (vc / kStages) & 1, kWhereVFull, t);
+        const int j = t & 1, sv = vc % kPVS;
+        ok = wait_all(V_FULL + sv, (vc / kPVS) & 1, kWhereVFull, t);
         if (!ok) break;
         ok = wait_all(P_FULL + 2 * j, used[j] & 1, kWherePFull, t);
         if (!ok) break;
