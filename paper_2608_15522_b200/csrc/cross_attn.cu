@@ -401,10 +401,21 @@ __global__ void __launch_bounds__(256) head_sum_kernel(const float* __restrict__
   const int64_t idx = static_cast<int64_t>(blockIdx.x) * 256 + threadIdx.x;
   if (idx >= static_cast<int64_t>(B) * Nk) return;
   const int b = static_cast<int>(idx / Nk), i = static_cast<int>(idx % Nk);
+  // Fixed summation order: head major, partial slot minor.  Eight loads are issued together (a plain loop made
+  // each thread wait for H dependent round trips), the adds stay in order.
+  const int J = H * NCH;
   float acc = 0.f;
-  for (int h = 0; h < H; h++)
-    for (int ch = 0; ch < NCH; ch++)
-      acc += partial[(static_cast<int64_t>(ch) * B * H + static_cast<int64_t>(b) * H + h) * Nk + i];
+  for (int j0 = 0; j0 < J; j0 += 8) {
+    float v[8];
+#pragma unroll
+    for (int u = 0; u < 8; u++) {
+      const int j = j0 + u, h = j / NCH, ch = j % NCH;
+      v[u] = (j < J) ? partial[(static_cast<int64_t>(ch) * B * H + static_cast<int64_t>(b) * H + h) * Nk + i] : 0.f;
+    }
+#pragma unroll
+    for (int u = 0; u < 8; u++)
+      if (j0 + u < J) acc += v[u];
+  }
   float out = gamma * acc;
   if (beta != 0.f) out = fmaf(beta, scores[idx], out);
   scores[idx] = out;
