@@ -6,10 +6,11 @@
 // fill, and at the end the drain, the staged store and the teardown.  With one CTA per SM (shared and tensor
 // memory are both used in full) nothing overlaps that time, and a 64-tile work item lasts only about 60 us.
 // Here the roles of attn_fast_kernel loop over work items instead:
-//   * warp 0 is scheduler and K producer: it takes the next item from a global counter (through an order
-//     array that puts the long lists first), checks its list, and publishes it in a two-slot ring one item ahead; its K ring simply continues into the next item's tiles,
-//     and Q of the next item is loaded as soon as the last Q K^T of the current one has been issued;
-//   * warp 3 (V), warp 1 (Q K^T) and warp 2 (P V) follow the published items; all ring positions and barrier
+//   * warp 3 is scheduler and V producer: it takes the next item from a global counter (through an order
+//     array that puts the long lists first), checks its list, and publishes it in a four-slot ring two items
+//     ahead of the one whose V tiles it is loading (V is needed last in a tile's life, so this warp has the slack);
+//   * warp 0 (Q and K), warp 1 (Q K^T) and warp 2 (P V) follow the published items; the K and V rings simply
+//     continue into the next item's tiles, Q alternates between two buffers, and all ring positions and barrier
 //     phases are running counts, not per-item indices;
 //   * the softmax groups finish an item by exchanging their row sums, reading the accumulator out of tensor
 //     memory (which hands it back to the P V warp for the next item) and writing their half rows straight to
@@ -21,9 +22,11 @@
 
 namespace avsa {
 
-// K stages, V stages, Q buffers.  Measured on the Ovi-class layer and on one-tile lists: (3,3,1), (3,2,2), (2,3,2),
-// (4,2,1) and (2,4,1) are all within noise of each other, so the simplest split of the 226 KB stays.
-constexpr int kPKS = 3, kPVS = 3, kPQB = 1;
+// K stages, V stages, Q buffers, slots of the item ring.  On the benchmark shapes (64-256 tiles per item) the splits
+// (3,3,1), (3,2,2), (2,3,2), (4,2,1) and (2,4,1) of the 226 KB are within noise of each other; the second Q buffer and
+// the deeper item ring are there for lists of a few tiles, where the next item's fetch and Q load would otherwise
+// sit in the critical path.
+constexpr int kPKS = 3, kPVS = 2, kPQB = 2, kPRing = 4;
 
 template <int BLK, int D>
 struct PersistSmem {
@@ -33,10 +36,10 @@ struct PersistSmem {
   static constexpr int kK = kPQB * kQBytes;
   static constexpr int kV = kK + kPKS * kTileBytes;
   static constexpr int kBars = kV + kPVS * kTileBytes;
-  static constexpr int kNumBars = 2 * kPQB + 2 * kPKS + 2 * kPVS + 21;
+  static constexpr int kNumBars = 2 * kPQB + 2 * kPKS + 2 * kPVS + 17 + 2 * kPRing;
   static constexpr int kStats = kBars + kNumBars * 8;          // float mref[128], lsum[2][128]
-  static constexpr int kItems = kStats + 3 * 128 * 4;          // int {item, cnt}[2], redo flag
-  static constexpr int kMisc = kItems + 32;                    // tmem base, stop flag
+  static constexpr int kItems = kStats + 3 * 128 * 4;          // int {item, cnt}[kPRing], redo flag
+  static constexpr int kMisc = kItems + 8 * kPRing + 16;       // tmem base, stop flag
   static constexpr int kTotal = kMisc + 16;
 };
 
@@ -100,15 +103,16 @@ attn_persist_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_consta
   constexpr int Q_FULL = 0, Q_EMPTY = kPQB, K_FULL = 2 * kPQB, K_EMPTY = K_FULL + kPKS, V_FULL = K_EMPTY + kPKS,
                 V_EMPTY = V_FULL + kPVS, S_FULL = V_EMPTY + kPVS /* + group */, S_FREE = S_FULL + 2,
                 P_FULL = S_FREE + 2 /* + 2*group + half */, P_FREE = P_FULL + 4, O_FULL = P_FREE + 2,
-                O_FREE = O_FULL + 1, MREF = O_FREE + 1, ITEM_FULL = MREF + 1 /* + slot */, ITEM_EMPTY = ITEM_FULL + 2,
-                QK_DRAIN = ITEM_EMPTY + 2, PV_DRAIN = QK_DRAIN + 1, LSUM_A = PV_DRAIN + 1, LSUM_B = LSUM_A + 1;
+                O_FREE = O_FULL + 1, MREF = O_FREE + 1, ITEM_FULL = MREF + 1 /* + slot */, ITEM_EMPTY = ITEM_FULL + kPRing,
+                QK_DRAIN = ITEM_EMPTY + kPRing, PV_DRAIN = QK_DRAIN + 1, LSUM_A = PV_DRAIN + 1, LSUM_B = LSUM_A + 1;
   static_assert(LSUM_B + 1 <= L::kNumBars, "barrier table too small");
   // tensor memory: S of group 0 | S of group 1 | O | P of group 0 | P of group 1
   constexpr uint32_t TM_O = 2 * BLK, TM_P = 2 * BLK + D;
   constexpr int NCH = BLK / 32;
   float* mref_s = reinterpret_cast<float*>(smem + L::kStats);
   float* lsum_s = mref_s + 128;                                              // [2][128]
-  volatile int* items = reinterpret_cast<volatile int*>(smem + L::kItems);   // {item, cnt} x 2, [4] = redo flag
+  volatile int* items = reinterpret_cast<volatile int*>(smem + L::kItems);   // {item, cnt} x kPRing, then the redo flag
+  constexpr int REDO = 2 * kPRing;
   volatile uint32_t* misc = reinterpret_cast<volatile uint32_t*>(smem + L::kMisc);   // [0] tmem base, [1] stop
 
   if (tid == 0) {
@@ -130,8 +134,10 @@ attn_persist_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_consta
       mbar_init(BAR(P_FULL + 2 * g), 128);
       mbar_init(BAR(P_FULL + 2 * g + 1), 128);
       mbar_init(BAR(P_FREE + g), 1);
-      mbar_init(BAR(ITEM_FULL + g), 1);
-      mbar_init(BAR(ITEM_EMPTY + g), 11);      // one arrival per consumer warp (all but the scheduler)
+    }
+    for (int r = 0; r < kPRing; r++) {
+      mbar_init(BAR(ITEM_FULL + r), 1);
+      mbar_init(BAR(ITEM_EMPTY + r), 11);      // one arrival per consumer warp (all but the scheduler)
     }
     mbar_init(BAR(O_FULL), 1);
     mbar_init(BAR(O_FREE), 256);
@@ -141,7 +147,7 @@ attn_persist_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_consta
     mbar_init(BAR(LSUM_A), 256);
     mbar_init(BAR(LSUM_B), 256);
     misc[1] = 0u;
-    items[4] = 0;
+    items[REDO] = 0;
     fence_mbar_init();
     prefetch_tmap(&tmq);
     prefetch_tmap(&tmk);
@@ -173,26 +179,85 @@ attn_persist_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_consta
   auto wait_all = [&](int bar, uint32_t parity, int where, int tag) -> bool {
     return __all_sync(FULLM, wait_or_stop(bar, parity, where, tag));
   };
-  // consumer side of the item ring: item n sits in slot n & 1
+  // consumer side of the item ring: item n sits in slot n mod kPRing
   auto get_item = [&](int n, int& item, int& cnt) -> bool {     // false: stopped, or the queue is empty
-    if (!wait_all(ITEM_FULL + (n & 1), (n >> 1) & 1, kPersistItem, n)) return false;
-    item = items[2 * (n & 1)];
-    cnt = items[2 * (n & 1) + 1];
+    const int slot = n % kPRing;
+    if (!wait_all(ITEM_FULL + slot, (n / kPRing) & 1, kPersistItem, n)) return false;
+    item = items[2 * slot];
+    cnt = items[2 * slot + 1];
     return item >= 0;
   };
   auto item_done = [&](int n) {
     __syncwarp();
-    if (lane == 0) mbar_arrive(BAR(ITEM_EMPTY + (n & 1)));
+    if (lane == 0) mbar_arrive(BAR(ITEM_EMPTY + n % kPRing));
   };
 
   if (warp == 0) {
-    // ------------------------------------------------------------------ scheduler + TMA producer of Q and K
+    // ------------------------------------------------------------------ TMA producer of Q and K
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 64;");
+    int kc = 0;              // K tiles loaded so far, over all items
+    int q_loads = 0;
+    bool ok = true;
+    for (int n = 0; ok; n++) {
+      int item, cnt;
+      if (!get_item(n, item, cnt)) break;
+      const PersistItem it = decode_item<MODE>(p, item);
+      const int qt = it.qt, h = it.h, b = it.b;
+      const int qb = n % kPQB;
+      if (n >= kPQB) {
+        // the last Q K^T of the item that used this Q buffer has run
+        ok = wait_all(Q_EMPTY + qb, ((n / kPQB) - 1) & 1, kPersistQEmpty, n);
+        if (!ok) break;
+      }
+      if (lane == 0) {
+        mbar_expect_tx(BAR(Q_FULL + qb), BLK * D * 2);
+        for (int pn = 0; pn < NPANEL; pn++)
+          tma_load_4d(smem_u32(smem + L::kQ) + qb * L::kQBytes + pn * QPANEL_BYTES, &tmq, BAR(Q_FULL + qb), pn * 64,
+                      qt * BLK, h, b);
+        q_loads++;
+      }
+      for (int t0 = 0; t0 < cnt && ok; t0 += 32) {
+        int mine = it.kb0 + t0 + lane;
+        if (kListIn) mine = (t0 + lane < cnt) ? it.list[t0 + lane] : 0;
+        const int nn = min(32, cnt - t0);
+        for (int j = 0; j < nn; j++) {
+          const int kb = __shfl_sync(FULLM, mine, j);
+          const int s = kc % kPKS;
+          int good = 1;
+          if (lane == 0) {
+            if (kc >= kPKS) good = wait_or_stop(K_EMPTY + s, ((kc / kPKS) - 1) & 1, kWhereKEmpty, t0 + j) ? 1 : 0;
+            if (good) {
+              mbar_expect_tx(BAR(K_FULL + s), L::kTileBytes);
+              for (int pn = 0; pn < NPANEL; pn++)
+                tma_load_4d(smem_u32(smem + L::kK) + s * L::kTileBytes + pn * PANEL_BYTES, &tmk, BAR(K_FULL + s), pn * 64,
+                            kb * BLK, h, b);
+            }
+          }
+          good = __shfl_sync(FULLM, good, 0);
+          if (!good) {
+            ok = false;
+            break;
+          }
+          kc++;
+        }
+      }
+      if (ok) item_done(n);
+    }
+    if (lane == 0 && misc[1] != 0u) {
+      // stopped: loads still in flight must land before this CTA's shared memory is given away
+      for (int c = max(0, q_loads - kPQB); c < q_loads; c++) mbar_wait(BAR(Q_FULL + c % kPQB), (c / kPQB) & 1);
+      for (int c = max(0, kc - kPKS); c < kc; c++) mbar_wait(BAR(K_FULL + c % kPKS), (c / kPKS) & 1);
+    }
+  } else if (warp == 3) {
+    // ------------------------------------------------------------------ scheduler + TMA producer of V
+    // V is needed last in a tile's life, so this warp has the slack to fetch work: it keeps the item ring two
+    // items ahead of the one whose V tiles it is loading.
     asm volatile("setmaxnreg.dec.sync.aligned.u32 64;");
     int pub_item = -1, pub_cnt = 0;
     // takes the next valid work item off the global queue and publishes it as item m of this CTA
     auto publish = [&](int m) -> bool {
-      const int slot = m & 1;
-      if (m >= 2 && !wait_all(ITEM_EMPTY + slot, ((m >> 1) - 1) & 1, kPersistItemEmpty, m)) return false;
+      const int slot = m % kPRing;
+      if (m >= kPRing && !wait_all(ITEM_EMPTY + slot, ((m / kPRing) - 1) & 1, kPersistItemEmpty, m)) return false;
       while (true) {
         int id = 0;
         if (lane == 0) id = atomicAdd(&p.status->next_item, 1);
@@ -240,83 +305,22 @@ attn_persist_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_consta
       __syncwarp();
       return true;
     };
-    int n = 0;
-    int kc = 0;              // K tiles loaded so far, over all items
-    int q_loads = 0;
+    int vc = 0;              // V tiles loaded so far, over all items
     bool ok = publish(0);
-    int cur_item = pub_item, cur_cnt = pub_cnt;
-    while (ok && cur_item >= 0) {
-      const PersistItem it = decode_item<MODE>(p, cur_item);
-      const int qt = it.qt, h = it.h, b = it.b;
-      const int qb = n % kPQB;
-      if (n >= kPQB) {
-        // the last Q K^T of the item that used this Q buffer has run
-        ok = wait_all(Q_EMPTY + qb, ((n / kPQB) - 1) & 1, kPersistQEmpty, n);
-        if (!ok) break;
-      }
-      if (lane == 0) {
-        mbar_expect_tx(BAR(Q_FULL + qb), BLK * D * 2);
-        for (int pn = 0; pn < NPANEL; pn++)
-          tma_load_4d(smem_u32(smem + L::kQ) + qb * L::kQBytes + pn * QPANEL_BYTES, &tmq, BAR(Q_FULL + qb), pn * 64,
-                      qt * BLK, h, b);
-        q_loads++;
-      }
-      const int pub_at = min(cur_cnt, kPKS) - 1;     // the next item is fetched once the K ring has been filled
-      int nxt_item = -1, nxt_cnt = 0;
-      for (int t0 = 0; t0 < cur_cnt && ok; t0 += 32) {
-        int mine = it.kb0 + t0 + lane;
-        if (kListIn) mine = (t0 + lane < cur_cnt) ? it.list[t0 + lane] : 0;
-        const int nn = min(32, cur_cnt - t0);
-        for (int j = 0; j < nn && ok; j++) {
-          const int kb = __shfl_sync(FULLM, mine, j);
-          const int t = t0 + j;
-          const int s = kc % kPKS;
-          int good = 1;
-          if (lane == 0) {
-            if (kc >= kPKS) good = wait_or_stop(K_EMPTY + s, ((kc / kPKS) - 1) & 1, kWhereKEmpty, t) ? 1 : 0;
-            if (good) {
-              mbar_expect_tx(BAR(K_FULL + s), L::kTileBytes);
-              for (int pn = 0; pn < NPANEL; pn++)
-                tma_load_4d(smem_u32(smem + L::kK) + s * L::kTileBytes + pn * PANEL_BYTES, &tmk, BAR(K_FULL + s), pn * 64,
-                            kb * BLK, h, b);
-            }
-          }
-          good = __shfl_sync(FULLM, good, 0);
-          if (!good) {
-            ok = false;
-            break;
-          }
-          kc++;
-          if (t == pub_at) {
-            ok = publish(n + 1);
-            nxt_item = pub_item;
-            nxt_cnt = pub_cnt;
-          }
-        }
-      }
-      cur_item = nxt_item;
-      cur_cnt = nxt_cnt;
-      n++;
+    int a_item = pub_item, a_cnt = pub_cnt;       // item n, whose V tiles are loaded next
+    int b_item = -1, b_cnt = 0;                   // item n + 1
+    if (ok && a_item >= 0) {
+      ok = publish(1);
+      b_item = pub_item;
+      b_cnt = pub_cnt;
     }
-    if (lane == 0 && misc[1] != 0u) {
-      // stopped: loads still in flight must land before this CTA's shared memory is given away
-      for (int c = max(0, q_loads - kPQB); c < q_loads; c++) mbar_wait(BAR(Q_FULL + c % kPQB), (c / kPQB) & 1);
-      for (int c = max(0, kc - kPKS); c < kc; c++) mbar_wait(BAR(K_FULL + c % kPKS), (c / kPKS) & 1);
-    }
-  } else if (warp == 3) {
-    // ------------------------------------------------------------------ TMA producer of V
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 64;");
-    int vc = 0;
-    bool ok = true;
-    for (int n = 0; ok; n++) {
-      int item, cnt;
-      if (!get_item(n, item, cnt)) break;
-      const PersistItem it = decode_item<MODE>(p, item);
+    for (int n = 0; ok && a_item >= 0; n++) {
+      const PersistItem it = decode_item<MODE>(p, a_item);
       const int h = it.h, b = it.b;
-      for (int t0 = 0; t0 < cnt && ok; t0 += 32) {
+      for (int t0 = 0; t0 < a_cnt && ok; t0 += 32) {
         int mine = it.kb0 + t0 + lane;
-        if (kListIn) mine = (t0 + lane < cnt) ? it.list[t0 + lane] : 0;
-        const int nn = min(32, cnt - t0);
+        if (kListIn) mine = (t0 + lane < a_cnt) ? it.list[t0 + lane] : 0;
+        const int nn = min(32, a_cnt - t0);
         for (int j = 0; j < nn; j++) {
           const int kb = __shfl_sync(FULLM, mine, j);
           const int s = vc % kPVS;
@@ -338,7 +342,18 @@ attn_persist_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_consta
           vc++;
         }
       }
-      if (ok) item_done(n);
+      if (!ok) break;
+      // keep the ring two items ahead (nothing more once the end of the queue has been published)
+      int c_item = -1, c_cnt = 0;
+      if (b_item >= 0) {
+        ok = publish(n + 2);
+        c_item = pub_item;
+        c_cnt = pub_cnt;
+      }
+      a_item = b_item;
+      a_cnt = b_cnt;
+      b_item = c_item;
+      b_cnt = c_cnt;
     }
     if (lane == 0 && misc[1] != 0u)
       for (int c = max(0, vc - kPVS); c < vc; c++) mbar_wait(BAR(V_FULL + c % kPVS), (c / kPVS) & 1);
@@ -543,19 +558,19 @@ attn_persist_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_consta
       }
       // A row sum beyond 2^64 (or not finite) means the row outgrew its first-tile reference: the item is left
       // to the exact-rescaling kernel.
-      if (!(l_run <= kFastRowSumLimit)) items[4] = 1;
+      if (!(l_run <= kFastRowSumLimit)) items[REDO] = 1;
       lsum_s[w * 128 + row] = l_run;
       // (time-limited barriers, not bar.sync: a group that gave up must not leave the other one waiting for ever)
       mbar_arrive(BAR(LSUM_A));
       ok = __all_sync(FULLM, wait_or_stop(LSUM_A, n & 1, kPersistLsum, n));
       if (!ok) break;
       const float Lsum = l_run + lsum_s[(1 - w) * 128 + row];
-      const bool redo = items[4] != 0;
+      const bool redo = items[REDO] != 0;
       mbar_arrive(BAR(LSUM_B));                           // everyone has read the sums and the flag
       ok = __all_sync(FULLM, wait_or_stop(LSUM_B, n & 1, kPersistLsum, n));
       if (!ok) break;
       if (tid == 128) {
-        items[4] = 0;
+        items[REDO] = 0;
         if (redo) redo_list[atomicAdd(&p.status->redo_count, 1)] = item;
       }
       ok = __all_sync(FULLM, wait_or_stop(O_FULL, n & 1, kPersistOFull, n));
