@@ -53,8 +53,6 @@ struct AttnParams {
   const int32_t* col_idx;   // [B,H,NB,NB]
   const int32_t* col_cnt;   // [B,H,NB]
   float* lse;               // [B,H,Nq] natural log, optional
-  __nv_bfloat16* o;         // output tensor and its element strides (kernels that store rows directly)
-  int64_t o_sb, o_sh, o_sn;
   // MODE_RANGE
   float* part_o;            // [items][BLK][D] fp32
   float* part_lse2;         // [items][BLK]
@@ -81,8 +79,8 @@ struct AttnParams {
 #endif
 
 // One work item of the tile kernel: query tile `bx` (MODE_LIST) or query tile / key split `bx`
-// (range modes) of head `by`, batch item `bz`.  Called once per CTA by attn_fwd_kernel and once per
-// flagged work item by attn_redo_kernel; every thread of the CTA must call it.
+// (range modes) of head `by`, batch item `bz`.  Called once per flagged work item by attn_redo_kernel;
+// every thread of the CTA must call it.
 template <int BLK, int D, int MODE>
 __device__ __forceinline__ void attn_fwd_body(const CUtensorMap* tmq, const CUtensorMap* tmk, const CUtensorMap* tmv,
                                               const CUtensorMap* tmo, const AttnParams& p, int bx, int by, int bz) {
@@ -482,14 +480,6 @@ __device__ __forceinline__ void attn_fwd_body(const CUtensorMap* tmq, const CUte
   tc_fence_before();
   __syncthreads();
   if (warp == 2) tmem_dealloc(tmem, 512);
-}
-
-template <int BLK, int D, int MODE>
-__global__ void __launch_bounds__(kAttnThreads, 1)
-attn_fwd_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUtensorMap tmk,
-                const __grid_constant__ CUtensorMap tmv, const __grid_constant__ CUtensorMap tmo,
-                const AttnParams p) {
-  attn_fwd_body<BLK, D, MODE>(&tmq, &tmk, &tmv, &tmo, p, blockIdx.x, blockIdx.y, blockIdx.z);
 }
 
 // Exact-rescaling pass behind the fast kernels: recomputes the work items they listed (normally none: then

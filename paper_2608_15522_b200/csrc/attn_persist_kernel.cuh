@@ -1,32 +1,48 @@
-// Persistent form of attn_fast_kernel: one CTA per SM walks a queue of work items (query tiles) and keeps
-// its pipeline running across them.
+// The fast attention tile kernel, in persistent form: one CTA per SM walks a queue of work items (query tiles)
+// and keeps its pipeline running across them.
 //
-// A CTA of attn_fast_kernel spends about 6 us outside its steady state: launch, barrier and tensor-memory
-// set-up, the first Q/K/V loads (about 3000 cycles of TMA latency with nothing to hide them behind), pipeline
-// fill, and at the end the drain, the staged store and the teardown.  With one CTA per SM (shared and tensor
-// memory are both used in full) nothing overlaps that time, and a 64-tile work item lasts only about 60 us.
-// Here the roles of attn_fast_kernel loop over work items instead:
-//   * warp 3 is scheduler and V producer: it takes the next item from a global counter (through an order
-//     array that puts the long lists first), checks its list, and publishes it in a four-slot ring two items
-//     ahead of the one whose V tiles it is loading (V is needed last in a tile's life, so this warp has the slack);
-//   * warp 0 (Q and K), warp 1 (Q K^T) and warp 2 (P V) follow the published items; the K and V rings simply
-//     continue into the next item's tiles, Q alternates between two buffers, and all ring positions and barrier
-//     phases are running counts, not per-item indices;
-//   * the softmax groups finish an item by exchanging their row sums, reading the accumulator out of tensor
-//     memory (which hands it back to the P V warp for the next item) and writing their half rows straight to
-//     global memory with 32-byte stores; the next item's first S tiles are already waiting by then.
-// Numerics, the fixed first-tile reference maximum and the hand-over of rows that outgrow it (redo_list)
-// are those of attn_fast_kernel.  Requires the output rows to be 32-byte aligned.
+// Against attn_fwd_body (the exact-rescaling kernel, where each softmax group owns one S buffer that P overwrites in
+// place and one accumulator that is rescaled when the row maximum grows, so that S for a group's next tile can only
+// be issued after the P V of its current tile):
+//   * every row keeps ONE reference maximum, the maximum of its first tile.  Probabilities are exp2(s*c - m_ref);
+//     they may exceed 1 for later tiles, which fp32 accumulation and bf16 P tolerate (same relative precision at
+//     any magnitude) as long as nothing overflows.  No per-tile maximum, no rescaling: both groups add into the
+//     same accumulator O and their row sums simply add up;
+//   * tensor memory is S0 | S1 | O | P0 | P1.  The groups take alternate key tiles, P has its own buffer: a group
+//     releases its S buffer the moment the tile is in registers, so Q K^T of its next tile runs under the
+//     exponentials of the current one, and it waits for the P V that read its previous P only at the first store
+//     of the new P;
+//   * two warps issue MMAs, one the Q K^T products and one the P V products: every MMA and every barrier wait
+//     costs the issuing thread tens of cycles, which one warp doing both would serialise;
+//   * a CTA that handles one query tile spends about 6 us outside its steady state (launch, barrier and tensor-
+//     memory set-up, about 3000 cycles of TMA latency for the first tiles with nothing to hide them behind,
+//     pipeline fill, drain, store, teardown), and with one CTA per SM nothing overlaps that.  So the roles loop
+//     over work items instead:
+//     - warp 3 is scheduler and V producer: it takes the next item from a global counter (through an order array
+//       that puts the long lists first), checks its list, and publishes it in a four-slot ring two items ahead of
+//       the one whose V tiles it is loading (V is needed last in a tile's life, so this warp has the slack);
+//     - warp 0 (Q and K), warp 1 (Q K^T) and warp 2 (P V) follow the published items; the K and V rings simply
+//       continue into the next item's tiles, and all ring positions and barrier phases are running counts;
+//     - the softmax groups finish an item by exchanging their row sums, reading the accumulator out of tensor
+//       memory (which hands it back to the P V warp for the next item) and staging their half rows for one TMA
+//       store (the fp32 partials of the range mode go straight to global memory with 32-byte stores); the next
+//       item's first S tiles are already waiting by then.
+// A row whose sum, relative to m_ref, ends above 2^64 (or not finite) outgrew its reference: its work item is
+// appended to `redo_list` (count in the status record) and attn_redo_kernel, a small grid launched behind this
+// kernel, recomputes the listed items with exact rescaling.  List validation and bounded waits as in attn_fwd_body.
 #pragma once
-#include "attn_fast_kernel.cuh"
+#include "attn_kernel.cuh"
 
 namespace avsa {
 
+// Largest row sum, relative to the first-tile reference maximum, that the fast path accepts (2^64).
+constexpr float kFastRowSumLimit = 1.8446744e19f;
+enum FastWhere { kFastSFree = 61, kFastPFree, kFastMref };
+
 // K stages, V stages, Q buffers, slots of the item ring.  On the benchmark shapes (64-256 tiles per item) the splits
-// (3,3,1), (3,2,2), (2,3,2), (4,2,1) and (2,4,1) of the 226 KB are within noise of each other; the second Q buffer and
-// the deeper item ring are there for lists of a few tiles, where the next item's fetch and Q load would otherwise
-// sit in the critical path.
-constexpr int kPKS = 3, kPVS = 2, kPQB = 2, kPRing = 4;
+// (3,3,1), (3,2,2), (2,3,2), (4,2,1) and (2,4,1) of the seven 32 KB tile slots are within noise of each other; the
+// seventh slot is the staging buffer of the output tile.
+constexpr int kPKS = 3, kPVS = 2, kPQB = 1, kPRing = 4;
 
 template <int BLK, int D>
 struct PersistSmem {
@@ -35,15 +51,16 @@ struct PersistSmem {
   static constexpr int kQ = 0;
   static constexpr int kK = kPQB * kQBytes;
   static constexpr int kV = kK + kPKS * kTileBytes;
-  static constexpr int kBars = kV + kPVS * kTileBytes;
-  static constexpr int kNumBars = 2 * kPQB + 2 * kPKS + 2 * kPVS + 17 + 2 * kPRing;
+  static constexpr int kStage = kV + kPVS * kTileBytes;         // output tile, 128-byte swizzled, for the TMA store
+  static constexpr int kBars = kStage + kQBytes;
+  static constexpr int kNumBars = 2 * kPQB + 2 * kPKS + 2 * kPVS + 18 + 2 * kPRing;
   static constexpr int kStats = kBars + kNumBars * 8;          // float mref[128], lsum[2][128]
   static constexpr int kItems = kStats + 3 * 128 * 4;          // int {item, cnt}[kPRing], redo flag
   static constexpr int kMisc = kItems + 8 * kPRing + 16;       // tmem base, stop flag
   static constexpr int kTotal = kMisc + 16;
 };
 
-enum PersistWhere { kPersistItem = 71, kPersistItemEmpty, kPersistQEmpty, kPersistOFull, kPersistOFree, kPersistLsum };
+enum PersistWhere { kPersistItem = 71, kPersistItemEmpty, kPersistQEmpty, kPersistOFull, kPersistOFree, kPersistLsum, kPersistStage };
 
 __device__ __forceinline__ void st_global_v8(void* ptr, const uint32_t (&r)[8]) {
   asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(ptr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]),
@@ -82,8 +99,8 @@ __device__ __forceinline__ PersistItem decode_item(const AttnParams& p, int item
 template <int BLK, int D, int MODE>
 __global__ void __launch_bounds__(kAttnThreads, 1)
 attn_persist_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ CUtensorMap tmk,
-                    const __grid_constant__ CUtensorMap tmv, const AttnParams p, int* __restrict__ redo_list,
-                    const int* __restrict__ order, int n_items) {
+                    const __grid_constant__ CUtensorMap tmv, const __grid_constant__ CUtensorMap tmo,
+                    const AttnParams p, int* __restrict__ redo_list, const int* __restrict__ order, int n_items) {
   using L = PersistSmem<BLK, D>;
   constexpr bool kListIn = (MODE == MODE_LIST);
   constexpr bool kDirectOut = (MODE != MODE_RANGE);
@@ -104,8 +121,9 @@ attn_persist_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_consta
                 V_EMPTY = V_FULL + kPVS, S_FULL = V_EMPTY + kPVS /* + group */, S_FREE = S_FULL + 2,
                 P_FULL = S_FREE + 2 /* + 2*group + half */, P_FREE = P_FULL + 4, O_FULL = P_FREE + 2,
                 O_FREE = O_FULL + 1, MREF = O_FREE + 1, ITEM_FULL = MREF + 1 /* + slot */, ITEM_EMPTY = ITEM_FULL + kPRing,
-                QK_DRAIN = ITEM_EMPTY + kPRing, PV_DRAIN = QK_DRAIN + 1, LSUM_A = PV_DRAIN + 1, LSUM_B = LSUM_A + 1;
-  static_assert(LSUM_B + 1 <= L::kNumBars, "barrier table too small");
+                QK_DRAIN = ITEM_EMPTY + kPRing, PV_DRAIN = QK_DRAIN + 1, LSUM_A = PV_DRAIN + 1, LSUM_B = LSUM_A + 1,
+                STAGE_FULL = LSUM_B + 1;
+  static_assert(STAGE_FULL + 1 <= L::kNumBars, "barrier table too small");
   // tensor memory: S of group 0 | S of group 1 | O | P of group 0 | P of group 1
   constexpr uint32_t TM_O = 2 * BLK, TM_P = 2 * BLK + D;
   constexpr int NCH = BLK / 32;
@@ -146,12 +164,14 @@ attn_persist_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_consta
     mbar_init(BAR(PV_DRAIN), 1);
     mbar_init(BAR(LSUM_A), 256);
     mbar_init(BAR(LSUM_B), 256);
+    mbar_init(BAR(STAGE_FULL), 256);
     misc[1] = 0u;
     items[REDO] = 0;
     fence_mbar_init();
     prefetch_tmap(&tmq);
     prefetch_tmap(&tmk);
     prefetch_tmap(&tmv);
+    if (kDirectOut) prefetch_tmap(&tmo);
   }
   if (warp == 2) {
     tmem_alloc(smem_u32(smem + L::kMisc), 512);
@@ -560,6 +580,9 @@ attn_persist_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_consta
       // to the exact-rescaling kernel.
       if (!(l_run <= kFastRowSumLimit)) items[REDO] = 1;
       lsum_s[w * 128 + row] = l_run;
+      // the staged output tile of the item before must have been read by its TMA store before anybody writes the
+      // staging buffer again; the thread that issued the store makes sure of it before it joins the barrier below
+      if (kDirectOut && tid == 128) tma_store_wait_read();
       // (time-limited barriers, not bar.sync: a group that gave up must not leave the other one waiting for ever)
       mbar_arrive(BAR(LSUM_A));
       ok = __all_sync(FULLM, wait_or_stop(LSUM_A, n & 1, kPersistLsum, n));
@@ -587,19 +610,34 @@ attn_persist_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_consta
       const int64_t grow = static_cast<int64_t>(qt) * BLK + row;
       const float inv = 1.0f / Lsum;
       if (kDirectOut) {
-        if (!redo && row < BLK && grow < p.Nq) {
-          // half a row per thread, 32 bytes per store: every store fills whole sectors
-          __nv_bfloat16* orow = p.o + b * p.o_sb + h * p.o_sh + grow * p.o_sn + w * HALF;
+        // The tile goes out through shared memory (128-byte swizzled) and one TMA store.  Rows written straight
+        // from registers, even as whole 32-byte sectors, kept these warps busy for about 2000 cycles per item
+        // (1024 sector requests at 256-byte stride); the store's read of the staging buffer is only waited for
+        // when the next item is about to write it.
+        if (row < BLK) {
+          uint8_t* stage = smem + L::kStage;
 #pragma unroll
-          for (int g = 0; g < HALF / 16; g++) {
-            uint32_t r[8];
-#pragma unroll
-            for (int i = 0; i < 8; i++)
-              r[i] = pack_bf16x2(__uint_as_float(o0[g * 16 + 2 * i]) * inv, __uint_as_float(o0[g * 16 + 2 * i + 1]) * inv);
-            st_global_v8(orow + g * 16, r);
+          for (int g = 0; g < HALF / 8; g++) {
+            const int col = w * HALF + g * 8;
+            const int panel = col >> 6, chunk = (col & 63) >> 3;
+            uint4 val;
+            val.x = pack_bf16x2(__uint_as_float(o0[g * 8 + 0]) * inv, __uint_as_float(o0[g * 8 + 1]) * inv);
+            val.y = pack_bf16x2(__uint_as_float(o0[g * 8 + 2]) * inv, __uint_as_float(o0[g * 8 + 3]) * inv);
+            val.z = pack_bf16x2(__uint_as_float(o0[g * 8 + 4]) * inv, __uint_as_float(o0[g * 8 + 5]) * inv);
+            val.w = pack_bf16x2(__uint_as_float(o0[g * 8 + 6]) * inv, __uint_as_float(o0[g * 8 + 7]) * inv);
+            *reinterpret_cast<uint4*>(stage + panel * QPANEL_BYTES + row * 128 + ((chunk ^ (row & 7)) << 4)) = val;
           }
-          if (w == 0 && p.lse != nullptr)
+          if (!redo && w == 0 && p.lse != nullptr && grow < p.Nq)
             p.lse[(static_cast<int64_t>(b) * p.H + h) * p.Nq + grow] = (m_ref + log2f(Lsum)) * 0.6931471805599453f;
+        }
+        fence_proxy_async();
+        mbar_arrive(BAR(STAGE_FULL));
+        if (tid == 128) {
+          if (wait_or_stop(STAGE_FULL, n & 1, kPersistStage, n) && !redo) {
+            for (int pn = 0; pn < NPANEL; pn++)
+              tma_store_4d(&tmo, smem_u32(smem + L::kStage) + pn * QPANEL_BYTES, pn * 64, qt * BLK, h, b);
+            tma_store_commit();
+          }
         }
       } else if (!redo && row < BLK) {
         // normalised fp32 partial of this split + its log2 LSE, for merge_splits_kernel
@@ -615,6 +653,7 @@ attn_persist_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_consta
       }
       item_done(n);
     }
+    if (kDirectOut && tid == 128) tma_store_wait_read();     // the last store has read the staging buffer
   }
   tc_fence_before();
   __syncthreads();

@@ -511,30 +511,16 @@ static int run_cross(int B, int H, int Nq, int Nk, const avsa_bf16_4d& q, const 
       // the whole key axis fits one work item (few keys): write O and the LSE directly, no partials to merge
       CUtensorMap to;
       if (!encode_bf16_tile_map(&to, o, B, H, Nq, D, q.stride_b, q.stride_h, q.stride_n, BLK)) return AVSA_ERR_CUDA;
-      if (cudaFuncSetAttribute(attn_fwd_kernel<BLK, D, MODE_RANGE_DIRECT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+      prm.lse = lse;
+      if (cudaFuncSetAttribute(attn_persist_kernel<BLK, D, MODE_RANGE_DIRECT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                               LP::kTotal) != cudaSuccess)
+        return AVSA_ERR_CUDA;
+      if (cudaFuncSetAttribute(attn_redo_kernel<BLK, D, MODE_RANGE_DIRECT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                L::kTotal) != cudaSuccess)
         return AVSA_ERR_CUDA;
-      prm.lse = lse;
-      prm.o = static_cast<__nv_bfloat16*>(o);
-      prm.o_sb = q.stride_b;
-      prm.o_sh = q.stride_h;
-      prm.o_sn = q.stride_n;
-      const bool rows_aligned32 = (reinterpret_cast<uintptr_t>(o) & 31u) == 0 && q.stride_b % 16 == 0 &&
-                                  q.stride_h % 16 == 0 && q.stride_n % 16 == 0;
-      if (rows_aligned32) {
-        if (cudaFuncSetAttribute(attn_persist_kernel<BLK, D, MODE_RANGE_DIRECT>,
-                                 cudaFuncAttributeMaxDynamicSharedMemorySize, LP::kTotal) != cudaSuccess)
-          return AVSA_ERR_CUDA;
-        if (cudaFuncSetAttribute(attn_redo_kernel<BLK, D, MODE_RANGE_DIRECT>,
-                                 cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal) != cudaSuccess)
-          return AVSA_ERR_CUDA;
-        attn_persist_kernel<BLK, D, MODE_RANGE_DIRECT><<<pgrid, kAttnThreads, LP::kTotal, st>>>(
-            tq, tk, tv, prm, redo, nullptr, static_cast<int>(items));
-        attn_redo_kernel<BLK, D, MODE_RANGE_DIRECT><<<pgrid, kAttnThreads, L::kTotal, st>>>(tq, tk, tv, to, prm, redo);
-      } else {
-        dim3 grid(c.NQT * c.n_split, H, B);
-        attn_fwd_kernel<BLK, D, MODE_RANGE_DIRECT><<<grid, kAttnThreads, L::kTotal, st>>>(tq, tk, tv, to, prm);
-      }
+      attn_persist_kernel<BLK, D, MODE_RANGE_DIRECT><<<pgrid, kAttnThreads, LP::kTotal, st>>>(
+          tq, tk, tv, to, prm, redo, nullptr, static_cast<int>(items));
+      attn_redo_kernel<BLK, D, MODE_RANGE_DIRECT><<<pgrid, kAttnThreads, L::kTotal, st>>>(tq, tk, tv, to, prm, redo);
     } else {
       if (cudaFuncSetAttribute(attn_persist_kernel<BLK, D, MODE_RANGE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                LP::kTotal) != cudaSuccess)
@@ -542,7 +528,7 @@ static int run_cross(int B, int H, int Nq, int Nk, const avsa_bf16_4d& q, const 
       if (cudaFuncSetAttribute(attn_redo_kernel<BLK, D, MODE_RANGE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                L::kTotal) != cudaSuccess)
         return AVSA_ERR_CUDA;
-      attn_persist_kernel<BLK, D, MODE_RANGE><<<pgrid, kAttnThreads, LP::kTotal, st>>>(tq, tk, tv, prm, redo, nullptr,
+      attn_persist_kernel<BLK, D, MODE_RANGE><<<pgrid, kAttnThreads, LP::kTotal, st>>>(tq, tk, tv, tq, prm, redo, nullptr,
                                                                                        static_cast<int>(items));
       attn_redo_kernel<BLK, D, MODE_RANGE><<<pgrid, kAttnThreads, L::kTotal, st>>>(tq, tk, tv, tq, prm, redo);
       const int total_rows = B * H * Nq;

@@ -141,7 +141,7 @@ static int run_protected(int B, int H, int N, int n_protect, const avsa_bf16_4d&
   int* redo = reinterpret_cast<int*>(ws + c.off_redo);
   const long long items = static_cast<long long>(B) * H * c.NQT * c.n_split;
   const int grid = persistent_grid(items);
-  attn_persist_kernel<BLK, D, MODE_RANGE><<<grid, kAttnThreads, LP::kTotal, st>>>(tq, tk, tv, prm, redo, nullptr,
+  attn_persist_kernel<BLK, D, MODE_RANGE><<<grid, kAttnThreads, LP::kTotal, st>>>(tq, tk, tv, tq, prm, redo, nullptr,
                                                                                   static_cast<int>(items));
   attn_redo_kernel<BLK, D, MODE_RANGE><<<grid, kAttnThreads, L::kTotal, st>>>(tq, tk, tv, tq, prm, redo);
   const int total_rows = B * H * c.n_pad;

@@ -68,31 +68,18 @@ static int launch_sparse_attn(int B, int H, int N, const avsa_bf16_4d& q, const 
   if (!encode_bf16_tile_map(&tk, k.ptr, B, H, N, D, k.stride_b, k.stride_h, k.stride_n, BLK)) return AVSA_ERR_CUDA;
   if (!encode_bf16_tile_map(&tv, v.ptr, B, H, N, D, v.stride_b, v.stride_h, v.stride_n, BLK)) return AVSA_ERR_CUDA;
   if (!encode_bf16_tile_map(&to, o, B, H, N, D, q.stride_b, q.stride_h, q.stride_n, BLK)) return AVSA_ERR_CUDA;
-  using LF = FastSmem<BLK, D>;
-  if (cudaFuncSetAttribute(attn_fast_kernel<BLK, D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           LF::kTotal) != cudaSuccess)
-    return AVSA_ERR_CUDA;
   if (cudaFuncSetAttribute(attn_redo_kernel<BLK, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kTotal) !=
       cudaSuccess)
     return AVSA_ERR_CUDA;
-  dim3 grid(prm.NQT, H, B);
-  // The fast kernel (persistent form when the rows allow it) first; it lists the (rare) work items whose rows
-  // outgrow its fixed reference maxima, and the exact-rescaling kernel behind it recomputes exactly those.
+  // The persistent fast kernel first; it lists the (rare) work items whose rows outgrow its fixed reference
+  // maxima, and the exact-rescaling kernel behind it recomputes exactly those.
   const long long items = static_cast<long long>(prm.NQT) * H * B;
-  // The persistent form stores rows with 32-byte accesses: it needs 32-byte-aligned rows.
-  const bool rows_aligned32 = (reinterpret_cast<uintptr_t>(o) & 31u) == 0 && q.stride_b % 16 == 0 &&
-                              q.stride_h % 16 == 0 && q.stride_n % 16 == 0;
-  if (rows_aligned32 && items <= 0x7fffffff) {
-    using LP = PersistSmem<BLK, D>;
-    if (cudaFuncSetAttribute(attn_persist_kernel<BLK, D, MODE_LIST>, cudaFuncAttributeMaxDynamicSharedMemorySize, LP::kTotal) !=
-        cudaSuccess)
-      return AVSA_ERR_CUDA;
-    const int pgrid = persistent_grid(items);
-    attn_persist_kernel<BLK, D, MODE_LIST><<<pgrid, kAttnThreads, LP::kTotal, st>>>(tq, tk, tv, prm, redo, redo + items,
-                                                                         static_cast<int>(items));
-  } else {
-    attn_fast_kernel<BLK, D><<<grid, kAttnThreads, LF::kTotal, st>>>(tq, tk, tv, to, prm, redo);
-  }
+  using LP = PersistSmem<BLK, D>;
+  if (cudaFuncSetAttribute(attn_persist_kernel<BLK, D, MODE_LIST>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           LP::kTotal) != cudaSuccess)
+    return AVSA_ERR_CUDA;
+  attn_persist_kernel<BLK, D, MODE_LIST><<<persistent_grid(items), kAttnThreads, LP::kTotal, st>>>(
+      tq, tk, tv, to, prm, redo, redo + items, static_cast<int>(items));
   const int redo_grid = persistent_grid(items);
   attn_redo_kernel<BLK, D><<<redo_grid, kAttnThreads, L::kTotal, st>>>(tq, tk, tv, to, prm, redo);
   return cudaGetLastError() == cudaSuccess ? AVSA_OK : AVSA_ERR_CUDA;
@@ -133,10 +120,6 @@ extern "C" int avsa_sparse_self_attn(int B, int H, int N, int d, int blk, avsa_b
   prm.col_idx = col_idx;
   prm.col_cnt = col_cnt;
   prm.lse = lse;
-  prm.o = static_cast<__nv_bfloat16*>(o_bf16);
-  prm.o_sb = q.stride_b;
-  prm.o_sh = q.stride_h;
-  prm.o_sn = q.stride_n;
   prm.status = static_cast<StatusRecord*>(ws);
   prm.H = H;
   prm.Nq = N;

@@ -347,9 +347,8 @@ def test_sparse_attention_random_shapes_and_lists(seed):
 
 
 def test_sparse_attention_rows_not_32_byte_aligned():
-    """Rows 272 bytes apart (d padded by 8 elements): 16-byte aligned, as the interface requires, but not
-    32-byte aligned, so the call takes the one-CTA-per-query-tile kernel with the staged TMA store instead
-    of the persistent kernel with its 32-byte row stores.  Same result either way."""
+    """Rows 272 bytes apart (d padded by 8 elements): 16-byte aligned, which is all the interface asks for (the
+    tile loads and the staged tile store go through tensor maps).  Same result as the contiguous layout, bit for bit."""
     w = wl.WORKLOADS["medium128"]
     q, k, v = wl.make_self_qkv(w, 12)
     NB = w.n_blocks
@@ -372,7 +371,7 @@ def test_sparse_attention_rows_not_32_byte_aligned():
     want_o, want_l = orc.masked_attention(_np64(q), _np64(k), _np64(v), idx, cnt, w.blk)
     _close(_np64(o), want_o, "padded rows O")
     _close(_np64(lse), want_l, "padded rows lse")
-    # and the aligned layout gives the same numbers bit for bit (both kernels share their arithmetic)
+    # and the contiguous layout gives the same numbers bit for bit
     o2, lse2, ws2 = av.avsa_sparse_self_attn(q.cuda(), k.cuda(), v.cuda(), torch.from_numpy(idx).cuda(),
                                              torch.from_numpy(cnt).cuda(), w.blk, want_lse=True)
     _status_ok(ws2)
