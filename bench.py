@@ -35,8 +35,8 @@ UNIT = "TFLOP/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the sparse attention kernel, from the ncu capture
 # summarised under profiles/ (None until a capture exists for that workload)
-NCU_TRAFFIC_BYTES = {"mid": 483.0e6,      # captured (profiles/attn_persist_kernel_mid.md)
-                     "ovi": 863.7e6}      # captured on the full launch with the two DRAM counters only (same file)
+NCU_TRAFFIC_BYTES = {"mid": 482.3e6,      # captured (profiles/attn_persist_kernel_mid.md)
+                     "ovi": 861.1e6}      # captured on the full launch with the two DRAM counters only (same file)
 KERNELS_PER_STEP = 12   # cross: clear, pass 1, merge, pass 2, head sum; mask: select, pool, scores, rows; attn: clear, persistent, redo
 
 
