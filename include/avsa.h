@@ -20,6 +20,12 @@
  *   - `ws` is scratch of at least the matching *_workspace_bytes(); its first 16 bytes are a status
  *     record the kernels fill when a device-side check fails (a wait that ran out of time, or a
  *     malformed column list).  Calls on the same workspace must not overlap on the GPU.
+ *   - The attention calls (cross-attention pass 1, sparse self-attention, protected rows) run a kernel that
+ *     normalises each row by the maximum of its first key tile instead of a running maximum (softmax is
+ *     invariant to that shift), and behind it an exact-rescaling kernel for the work items whose rows
+ *     outgrew that reference (a row whose sum of exp(logit - reference) ends above 2^64 or not finite;
+ *     values of v are assumed to stay below 2^60 in magnitude).  Results do not depend on which kernel
+ *     produced them beyond rounding; the int32 at byte 16 of ws counts the recomputed items (diagnostic).
  *   - Errors detectable on the host return at once with nothing enqueued.  Return values are
  *     avsa_status codes.
  *   - Supported shapes: (blk, d) in {(128,128), (64,64)}; any N >= 1 (the last block may be partial:
@@ -129,13 +135,9 @@ AVSA_API size_t avsa_build_block_mask_workspace_bytes(int B, int H, int N, int d
  * entry sets AVSA_ERR_BAD_MASK in the status record and that block is skipped without any
  * out-of-range access.  o is bf16 with the strides of q; lse (optional) is fp32 [B,H,N] natural log.
  *
- * Two kernels run: a fast one that keeps each row's first-tile maximum as the softmax reference (no
- * rescaling of the accumulator), and behind it the exact-rescaling kernel for the work items the fast
- * one had to give up (a row whose sum of exp(logit - reference) ends above 2^64 or is not finite; values of
- * v are assumed to stay below 2^60 in magnitude).
- * After the call the int32 at byte 16 of ws is the number of work items the exact kernel recomputed, and
- * their indices ((b*H + h)*NB + query block, in no particular order) follow as int32 behind the first
- * AVSA_STATUS_BYTES bytes (diagnostic; results do not depend on it).
+ * After the call the int32 at byte 16 of ws is the number of work items the exact kernel recomputed (see
+ * the conventions above), and their indices ((b*H + h)*NB + query block, in no particular order) follow
+ * as int32 behind the first AVSA_STATUS_BYTES bytes (diagnostic; results do not depend on it).
  */
 AVSA_API int avsa_sparse_self_attn(int B, int H, int N, int d, int blk, avsa_bf16_4d q, avsa_bf16_4d k, avsa_bf16_4d v,
                           const int32_t* col_idx, const int32_t* col_cnt, void* o_bf16, float* lse,
