@@ -112,6 +112,25 @@ def protected_blocks(prot_tok, blk, min_tokens=1):
     return out
 
 
+def protected_blocks_by_sum(s, blk, n_blocks):
+    """Variant of the block lift (not in the paper): protect the ``n_blocks`` blocks with the largest summed
+    response, ties to the lowest block index.  The sum of a block is taken in fp64 and rounded to fp32, and the
+    ranking is decided on that fp32 value.  s [B,N] -> uint8 [B,NB]."""
+    s = np.asarray(s, np.float64)
+    B, N = s.shape
+    nb = (N + blk - 1) // blk
+    out = np.zeros((B, nb), np.uint8)
+    for b in range(B):
+        sums = np.zeros(nb, np.float64)
+        for j in range(nb):
+            acc = 0.0
+            for i in range(j * blk, min((j + 1) * blk, N)):
+                acc += s[b, i]
+            sums[j] = acc
+        out[b, topk_indices(sums.astype(np.float32), n_blocks)] = 1
+    return out
+
+
 # ------------------------------------------------------------------------------------------------
 # base sparse pattern S_m (this build's rule; the paper leaves it open)
 # ------------------------------------------------------------------------------------------------
@@ -181,15 +200,23 @@ def keep_to_lists(keep):
 
 
 def build_block_mask(bs, scores, n_protect, k_keep, blk, n_tokens, protect_rows=True, protect_cols=False,
-                     min_tokens=1):
+                     min_tokens=1, block_sum=False):
     """Block scores + token scores -> (col_idx, col_cnt, prot_tok, prot_blk), the whole mask step."""
     bs = np.asarray(bs)
     B = bs.shape[0]
-    if n_protect > 0:
-        prot_tok = protected_tokens(scores, n_protect)
+    if block_sum:
+        # n_protect counts BLOCKS here; every token of a protected block is flagged
+        if n_protect > 0:
+            prot_blk = protected_blocks_by_sum(scores, blk, n_protect)
+        else:
+            prot_blk = np.zeros((B, (n_tokens + blk - 1) // blk), np.uint8)
+        prot_tok = np.repeat(prot_blk, blk, axis=1)[:, :n_tokens].astype(np.uint8)
     else:
-        prot_tok = np.zeros((B, n_tokens), np.uint8)
-    prot_blk = protected_blocks(prot_tok, blk, min_tokens)
+        if n_protect > 0:
+            prot_tok = protected_tokens(scores, n_protect)
+        else:
+            prot_tok = np.zeros((B, n_tokens), np.uint8)
+        prot_blk = protected_blocks(prot_tok, blk, min_tokens)
     keep = apply_protection(topk_blocks(bs, k_keep), prot_blk, protect_rows, protect_cols)
     idx, cnt = keep_to_lists(keep)
     return idx, cnt, prot_tok, prot_blk

@@ -185,6 +185,24 @@ def test_protected_blocks_lift():
     assert orc.protected_blocks(flags, 4, min_tokens=4).tolist() == [[0, 0, 0]]
 
 
+def test_protected_blocks_by_sum():
+    """Hand example: block sums 6 | 6 | 1.5 (two-token tail): the best block is block 0 (tie with block 1, lowest
+    index first), the best two are blocks 0 and 1; a NaN block ranks last."""
+    s = np.array([[1, 2, 3, 0, 6, 0, 0, 0, 1, 0.5]], np.float32)
+    assert orc.protected_blocks_by_sum(s, 4, 1).tolist() == [[1, 0, 0]]
+    assert orc.protected_blocks_by_sum(s, 4, 2).tolist() == [[1, 1, 0]]
+    assert orc.protected_blocks_by_sum(s, 4, 3).tolist() == [[1, 1, 1]]
+    s[0, 1] = np.nan
+    assert orc.protected_blocks_by_sum(s, 4, 1).tolist() == [[0, 1, 0]]
+    assert orc.protected_blocks_by_sum(s, 4, 2).tolist() == [[0, 1, 1]]
+    # through the whole mask step: all tokens of the chosen blocks are flagged, their rows are dense
+    bs = np.zeros((1, 1, 3, 3), np.float32); bs[0, 0] = np.eye(3)
+    s = np.array([[1, 2, 3, 0, 6, 0, 0, 0, 1, 0.5]], np.float32)
+    idx, cnt, ptok, pblk = orc.build_block_mask(bs, s, 1, 1, 4, 10, block_sum=True)
+    assert pblk.tolist() == [[1, 0, 0]] and ptok.tolist() == [[1, 1, 1, 1, 0, 0, 0, 0, 0, 0]]
+    assert cnt[0, 0].tolist() == [3, 1, 1] and idx[0, 0, 1].tolist() == [1, -1, -1]
+
+
 # ------------------------------------------------------------------------------- pooling, scores
 def test_block_mean_pool_closed_forms():
     B, H, N, d, blk = 1, 2, 11, 3, 4                                 # tail block of 3 tokens
