@@ -73,6 +73,11 @@ typedef struct {
 #define AVSA_PROTECT_TOKENS 8u          /* lists carry the base pattern only (no block is made dense); the
                                            protected rows are restored by avsa_protected_rows_attn */
 
+#define AVSA_PROTECT_BLOCK_SUM 16u      /* not in the paper: n_protect counts BLOCKS (0..NB); the protected blocks are
+                                           those with the largest summed response (fp64 sum of the block's scores
+                                           rounded to fp32, ties to the lowest block index); prot_tok flags every
+                                           token of a protected block.  Combines with ROWS / COLS / TOKENS. */
+
 /* Optional, ORed into flags: a block counts as protected only if it holds at least n (1..blk) protected tokens.
  * Not in the paper: in raster order a compact region straddles many blocks, and n > 1 trades the protection of
  * stray tokens for fewer dense blocks.  n = 0 or 1 is the block lift of Eq. 9 (any protected token). */

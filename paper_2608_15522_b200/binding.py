@@ -27,6 +27,7 @@ AVSA_PROTECT_ROWS = 1
 AVSA_PROTECT_COLS = 2
 AVSA_USE_GIVEN_BLOCK_SCORES = 4
 AVSA_PROTECT_TOKENS = 8
+AVSA_PROTECT_BLOCK_SUM = 16
 
 
 def AVSA_MIN_TOKENS_PER_BLOCK(n: int) -> int:

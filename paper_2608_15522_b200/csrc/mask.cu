@@ -450,8 +450,38 @@ __global__ void __launch_bounds__(128) row_select_kernel(const float* __restrict
   if (lane == 0) col_cnt[row] = pos;
 }
 
+// ------------------------------------------------------------------------------------------------
+// Optional block-sum protection (AVSA_PROTECT_BLOCK_SUM): the response of a block is the sum of its tokens'
+// scores, accumulated in fp64 (for 128 fp32 terms of like magnitude that sum is exact, so its value does not
+// depend on the order of the adds) and rounded to fp32; the top-n blocks are then chosen by the same select
+// kernel that chooses tokens.  One warp per block.
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) block_sum_kernel(const float* __restrict__ scores, int N, int blk, int NB,
+                                                        float* __restrict__ bsum) {
+  const int b = blockIdx.y, lane = threadIdx.x & 31;
+  const int j = blockIdx.x * 8 + (threadIdx.x >> 5);
+  if (j >= NB) return;
+  const float* s = scores + static_cast<int64_t>(b) * N;
+  const int lo = j * blk, hi = min(N, lo + blk);
+  double acc = 0.0;
+  for (int i = lo + lane; i < hi; i += 32) acc += static_cast<double>(__ldg(s + i));
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+  if (lane == 0) bsum[static_cast<int64_t>(b) * NB + j] = static_cast<float>(acc);
+}
+
+// prot_tok[b,i] = prot_blk[b, i / blk]
+__global__ void __launch_bounds__(256) expand_blocks_kernel(const uint8_t* __restrict__ prot_blk, int N, int blk, int NB,
+                                                            int64_t total, uint8_t* __restrict__ prot_tok) {
+  const int64_t idx = static_cast<int64_t>(blockIdx.x) * 256 + threadIdx.x;
+  if (idx >= total) return;
+  const int64_t b = idx / N;
+  const int i = static_cast<int>(idx % N);
+  prot_tok[idx] = prot_blk[b * NB + i / blk];
+}
+
 struct MaskWorkspace {
-  size_t qbar, kbar, ptok, pblk, total;
+  size_t qbar, kbar, ptok, pblk, bsum, junk, total;
 };
 static MaskWorkspace mask_ws_layout(int B, int H, int N, int d, int blk) {
   MaskWorkspace w;
@@ -461,6 +491,8 @@ static MaskWorkspace mask_ws_layout(int B, int H, int N, int d, int blk) {
   w.kbar = off; off += align_up(static_cast<size_t>(B) * H * NB * d * sizeof(float), 256);
   w.ptok = off; off += align_up(static_cast<size_t>(B) * N, 256);
   w.pblk = off; off += align_up(static_cast<size_t>(B) * NB, 256);
+  w.bsum = off; off += align_up(static_cast<size_t>(B) * NB * sizeof(float), 256);      // block-sum protection only
+  w.junk = off; off += align_up(static_cast<size_t>(B) * ((NB + 31) / 32), 256);
   w.total = off;
   return w;
 }
@@ -483,6 +515,8 @@ extern "C" int avsa_build_block_mask(int B, int H, int N, int d, int blk, avsa_b
   const int NB = (N + blk - 1) / blk;
   if (NB > kMaxBlocksPerRow) return AVSA_ERR_UNSUPPORTED;
   if (k_keep < 1 || k_keep > NB || n_protect < 0 || n_protect > N) return AVSA_ERR_INVALID_ARG;
+  const bool by_block_sum = (flags & AVSA_PROTECT_BLOCK_SUM) != 0;      // n_protect counts blocks
+  if (by_block_sum && n_protect > NB) return AVSA_ERR_INVALID_ARG;
   if (block_scores == nullptr || col_idx == nullptr || col_cnt == nullptr) return AVSA_ERR_INVALID_ARG;
   if (n_protect > 0 && scores == nullptr) return AVSA_ERR_INVALID_ARG;
   const bool given = (flags & AVSA_USE_GIVEN_BLOCK_SCORES) != 0;
@@ -500,7 +534,18 @@ extern "C" int avsa_build_block_mask(int B, int H, int N, int d, int blk, avsa_b
   uint8_t* pblk = prot_blk != nullptr ? prot_blk : base + w.pblk;
   const float scale = softmax_scale != 0.f ? softmax_scale : 1.0f / sqrtf(static_cast<float>(d));
 
-  if (N <= kSelectSmemKeys) {
+  if (by_block_sum) {
+    // block sums, then the token select run over the NB sums: its "token" flags are the block flags (its own
+    // block lift goes to a scratch array); the token flags are filled in at the end of the call
+    float* bsum = reinterpret_cast<float*>(base + w.bsum);
+    if (n_protect > 0) block_sum_kernel<<<dim3((NB + 7) / 8, B), 256, 0, st>>>(scores, N, blk, NB, bsum);
+    const size_t key_bytes = static_cast<size_t>(NB) * sizeof(uint32_t);
+    if (cudaFuncSetAttribute(token_select_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             static_cast<int>(key_bytes)) != cudaSuccess)
+      return AVSA_ERR_CUDA;
+    token_select_kernel<true><<<B, 1024, key_bytes, st>>>(bsum, NB, n_protect, 32, (NB + 31) / 32, 1, pblk,
+                                                         base + w.junk, static_cast<StatusRecord*>(ws));
+  } else if (N <= kSelectSmemKeys) {
     const size_t key_bytes = static_cast<size_t>(N) * sizeof(uint32_t);
     if (cudaFuncSetAttribute(token_select_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              static_cast<int>(key_bytes)) != cudaSuccess)
@@ -580,6 +625,10 @@ extern "C" int avsa_build_block_mask(int B, int H, int N, int d, int blk, avsa_b
     else
       e = cudaLaunchKernelEx(&rcfg, row_select_kernel<64>, bsc, pbc, H, NB, k_keep, pr, pc, total_rows, col_idx, col_cnt);
     if (e != cudaSuccess) return AVSA_ERR_CUDA;
+  }
+  if (by_block_sum) {
+    const int64_t total = static_cast<int64_t>(B) * N;
+    expand_blocks_kernel<<<static_cast<unsigned>((total + 255) / 256), 256, 0, st>>>(pblk, N, blk, NB, total, ptok);
   }
   return cudaGetLastError() == cudaSuccess ? AVSA_OK : AVSA_ERR_CUDA;
 }

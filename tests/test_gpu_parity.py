@@ -102,6 +102,32 @@ def test_mask_min_tokens_per_block_bit_exact(name, min_tokens):
     assert np.array_equal(out["col_idx"].cpu().numpy(), idx)
 
 
+@pytest.mark.parametrize("name,n_blocks,extra", [("tiny", 1, 0), ("medium128", 3, 0), ("medium128", 5, 2),
+                                                 ("medium128", 0, 0), ("medium128", 17, 0)])
+def test_mask_block_sum_protection_bit_exact(name, n_blocks, extra):
+    """Protected blocks = the n blocks with the largest summed response (flag AVSA_PROTECT_BLOCK_SUM), also with
+    key-column protection on top (extra = AVSA_PROTECT_COLS).  Block flags, token flags and lists bit-exact."""
+    w = wl.WORKLOADS[name]
+    _, _, _, s64 = _oracle_scores(w, 0)
+    q, k, _ = wl.make_self_qkv(w, 0)
+    k_keep = max(1, orc.ceil_pct(w.keep_pct, w.n_blocks))
+    bs32 = orc.block_scores(_np64(q), _np64(k), w.blk).astype(np.float32)
+    s32 = s64.astype(np.float32)
+    s32[:, 5] = np.nan                                   # a NaN score poisons its block's sum: that block ranks last
+    idx, cnt, ptok, pblk = orc.build_block_mask(bs32, s32, n_blocks, k_keep, w.blk, w.n_video, True, bool(extra),
+                                                block_sum=True)
+    assert pblk.sum() == n_blocks * w.B and (n_blocks == w.n_blocks or pblk[:, 0].sum() == 0)
+    out = av.avsa_build_block_mask(None, None, torch.from_numpy(s32).cuda(), n_blocks, k_keep, w.blk,
+                                   flags=av.AVSA_PROTECT_ROWS | extra | av.AVSA_USE_GIVEN_BLOCK_SCORES |
+                                   av.AVSA_PROTECT_BLOCK_SUM,
+                                   block_scores=torch.from_numpy(bs32).cuda(), shape=(w.B, w.H, w.n_video, w.d))
+    _status_ok(out["ws"])
+    assert np.array_equal(out["prot_blk"].cpu().numpy(), pblk)
+    assert np.array_equal(out["prot_tok"].cpu().numpy(), ptok)
+    assert np.array_equal(out["col_cnt"].cpu().numpy(), cnt)
+    assert np.array_equal(out["col_idx"].cpu().numpy(), idx)
+
+
 def test_mask_ties_nan_and_signed_zero_bit_exact():
     B, H, N, d, blk = 2, 2, 64 * 37 + 5, 64, 64
     NB = (N + blk - 1) // blk
