@@ -577,8 +577,9 @@ attn_persist_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_consta
         l_run = sa + sb;
       }
       // A row sum beyond 2^64 (or not finite) means the row outgrew its first-tile reference: the item is left
-      // to the exact-rescaling kernel.
-      if (!(l_run <= kFastRowSumLimit)) items[REDO] = 1;
+      // to the exact-rescaling kernel.  (With 64-row tiles the upper 64 lanes hold no rows: the 128-row MMA filled
+      // them from whatever follows the Q tile in shared memory, and their sums mean nothing.)
+      if (row < BLK && !(l_run <= kFastRowSumLimit)) items[REDO] = 1;
       lsum_s[w * 128 + row] = l_run;
       // the staged output tile of the item before must have been read by its TMA store before anybody writes the
       // staging buffer again; the thread that issued the store makes sure of it before it joins the barrier below

@@ -562,6 +562,7 @@ def test_whole_path_tiny_matches_oracle():
     m = av.avsa_build_block_mask(q, k, s, n_protect, k_keep, w.blk)
     o, _, ws = av.avsa_sparse_self_attn(q, k, v, m["col_idx"], m["col_cnt"], w.blk)
     _status_ok(ws)
+    assert av.avsa_redo_count(ws) == 0            # unit-variance logits never outgrow the first-tile reference
     # oracle end to end
     _, _, A = orc.cross_attention(_np64(qa), _np64(kc), _np64(vc))
     s64 = orc.column_scores(A, gamma=1.0 / (w.H * w.n_audio))
@@ -575,6 +576,67 @@ def test_whole_path_tiny_matches_oracle():
     assert np.array_equal(m["col_idx"].cpu().numpy(), idx)
     want, _ = orc.masked_attention(_np64(q), _np64(k), _np64(v), idx, cnt, w.blk)
     _close(_np64(o), want, "whole path O")
+
+
+@pytest.mark.parametrize("name", ["tiny", "medium128"])
+def test_whole_path_replays_from_a_cuda_graph(name):
+    """The calls only enqueue work on the given stream (no allocation, no synchronisation, no host read of
+    device data), so one layer-step can be captured into a CUDA graph once and replayed on new inputs.
+    The replays must reproduce the eager results bit for bit, and the eager results are held to the oracle."""
+    w = wl.WORKLOADS[name]
+    n_protect = av.avsa_count_from_percent(w.protect_pct, w.n_video)
+    k_keep = av.avsa_count_from_percent(w.keep_pct, w.n_blocks)
+    gamma = 1.0 / (w.H * w.n_audio)
+
+    def inputs(seed):
+        return [t.cuda() for t in wl.make_cross_qkv(w, seed)] + [t.cuda() for t in wl.make_self_qkv(w, seed)]
+
+    def eager(qa, kc, vc, q, k, v):
+        _, _, s, _ = av.avsa_cross_attn_scores(qa, kc, vc, score_gamma=gamma, want_o=False)
+        m = av.avsa_build_block_mask(q, k, s, n_protect, k_keep, w.blk)
+        o, lse, ws = av.avsa_sparse_self_attn(q, k, v, m["col_idx"], m["col_cnt"], w.blk, want_lse=True)
+        _status_ok(ws)
+        return s, m, o, lse
+
+    static = [t.clone() for t in inputs(0)]
+    qa, kc, vc, q, k, v = static
+    s0, m0, o0, lse0 = eager(*static)                       # also the warm-up that loads every kernel
+    # caller-owned buffers of the captured step
+    s = torch.empty_like(s0)
+    lse_a = torch.empty((w.B, w.H, w.n_audio), dtype=torch.float32, device="cuda")
+    out = {key: torch.empty_like(m0[key]) for key in ("block_scores", "col_idx", "col_cnt", "prot_tok", "prot_blk")}
+    o, lse = torch.empty_like(o0), torch.empty_like(lse0)
+    ws_c = torch.empty(av.avsa_cross_attn_scores_workspace_bytes(w.B, w.H, w.n_audio, w.n_video, w.d), dtype=torch.uint8, device="cuda")
+    ws_m = torch.empty(av.avsa_build_block_mask_workspace_bytes(w.B, w.H, w.n_video, w.d, w.blk), dtype=torch.uint8, device="cuda")
+    ws_a = torch.empty(av.avsa_sparse_self_attn_workspace_bytes(w.B, w.H, w.n_video, w.d, w.blk), dtype=torch.uint8, device="cuda")
+    graph = torch.cuda.CUDAGraph()
+    torch.cuda.synchronize()
+    with torch.cuda.graph(graph):
+        av.avsa_cross_attn_scores(qa, kc, vc, scores=s, score_gamma=gamma, want_o=False, lse=lse_a, ws=ws_c)
+        av.avsa_build_block_mask(q, k, s, n_protect, k_keep, w.blk, out=out, ws=ws_m)
+        av.avsa_sparse_self_attn(q, k, v, out["col_idx"], out["col_cnt"], w.blk, o=o, lse=lse, ws=ws_a)
+    for seed in (0, 5, 0):
+        fresh = inputs(seed)
+        for dst, src in zip(static, fresh):
+            dst.copy_(src)
+        for t in (s, o, lse, out["col_idx"], out["col_cnt"]):
+            t.fill_(0)
+        graph.replay()
+        torch.cuda.synchronize()
+        for ws_x in (ws_c, ws_m, ws_a):
+            _status_ok(ws_x)
+        assert av.avsa_redo_count(ws_a) == 0
+        want_s, want_m, want_o, want_lse = eager(*fresh)
+        assert torch.equal(s, want_s), f"seed {seed}: scores differ between replay and eager call"
+        for key in ("col_idx", "col_cnt", "prot_tok", "prot_blk", "block_scores"):
+            assert torch.equal(out[key], want_m[key]), f"seed {seed}: {key} differs between replay and eager call"
+        assert torch.equal(o.view(torch.int16), want_o.view(torch.int16)), f"seed {seed}: O differs"
+        assert torch.equal(lse, want_lse), f"seed {seed}: LSE differs"
+    # the eager results of the last seed against the oracle
+    idx, cnt = out["col_idx"].cpu().numpy(), out["col_cnt"].cpu().numpy()
+    want, want_l = orc.masked_attention(_np64(q), _np64(k), _np64(v), idx, cnt, w.blk)
+    _close(_np64(o), want, "graph replay O")
+    _close(_np64(lse), want_l, "graph replay lse")
 
 
 # ------------------------------------------------------------------------------------------- token-exact protection
