@@ -16,7 +16,9 @@
  *   - Tensors are bf16 with the head dimension contiguous, described by element strides (avsa_bf16_4d),
  *     so both [B,H,N,d] and [B,N,H,d] storage work.  Base pointers must be 16-byte aligned and strides
  *     multiples of 8 elements.
- *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  No call reads device
+ *     data on the host, so the calls may be recorded into a CUDA graph by stream capture (not on the legacy
+ *     default stream) and replayed; pointers, sizes and counts are fixed at capture time.
  *   - `ws` is scratch of at least the matching *_workspace_bytes(); its first 16 bytes are a status
  *     record the kernels fill when a device-side check fails (a wait that ran out of time, or a
  *     malformed column list).  Calls on the same workspace must not overlap on the GPU.
