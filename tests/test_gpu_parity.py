@@ -789,3 +789,70 @@ def test_host_side_argument_errors():
     with pytest.raises(av.AvsaError) as e:
         av.avsa_build_block_mask(q, k, None, 0, NB + 1, w.blk)
     assert e.value.status == av.AVSA_ERR_INVALID_ARG
+
+
+# ------------------------------------------------------------------------------------------- caller-owned scratch
+@pytest.mark.parametrize("name", ["tiny", "medium128"])
+def test_results_do_not_depend_on_what_the_buffers_held_before(name):
+    """Workspaces and outputs are caller-owned and arrive with arbitrary contents: every call must produce the
+    same bits whether they were zero-filled or filled with 0xFF bytes (NaN patterns, negative counts)."""
+    w = wl.WORKLOADS[name]
+    qa, kc, vc = (t.cuda() for t in wl.make_cross_qkv(w, 3))
+    q, k, v = (t.cuda() for t in wl.make_self_qkv(w, 3))
+    n_protect = av.avsa_count_from_percent(w.protect_pct, w.n_video)
+    k_keep = av.avsa_count_from_percent(w.keep_pct, w.n_blocks)
+    NB = w.n_blocks
+    C = w.H * w.d
+    g = torch.Generator().manual_seed(9)
+    y_v = torch.randn((w.B, w.n_video, C), generator=g).bfloat16().cuda()
+    yhat_v = (y_v.float() * 1.1).bfloat16()
+    y_a = torch.randn((w.B, w.n_audio, C), generator=g).bfloat16().cuda()
+    yhat_a = (y_a.float() * 0.9).bfloat16()
+
+    def run(fill):
+        def buf(shape, dtype):
+            t = torch.empty(shape, dtype=dtype, device="cuda")
+            t.view(torch.uint8).fill_(fill)
+            return t
+
+        def scratch(nbytes):
+            return buf((max(int(nbytes), 256),), torch.uint8)
+
+        res = {}
+        o_a, lse_a, s = buf(qa.shape, torch.bfloat16), buf(qa.shape[:3], torch.float32), buf((w.B, w.n_video), torch.float32)
+        ws = scratch(av.avsa_cross_attn_scores_workspace_bytes(w.B, w.H, w.n_audio, w.n_video, w.d))
+        av.avsa_cross_attn_scores(qa, kc, vc, scores=s, score_beta=0.0, score_gamma=1.0 / (w.H * w.n_audio), o=o_a,
+                                  lse=lse_a, ws=ws)
+        _status_ok(ws)
+        res.update(o_a=o_a, lse_a=lse_a, s=s)
+        for tag, flags in (("rows", av.AVSA_PROTECT_ROWS), ("tok", av.AVSA_PROTECT_TOKENS),
+                           ("sum", av.AVSA_PROTECT_ROWS | av.AVSA_PROTECT_BLOCK_SUM)):
+            out = dict(block_scores=buf((w.B, w.H, NB, NB), torch.float32), col_idx=buf((w.B, w.H, NB, NB), torch.int32),
+                       col_cnt=buf((w.B, w.H, NB), torch.int32), prot_tok=buf((w.B, w.n_video), torch.uint8),
+                       prot_blk=buf((w.B, NB), torch.uint8))
+            ws = scratch(av.avsa_build_block_mask_workspace_bytes(w.B, w.H, w.n_video, w.d, w.blk))
+            n = n_protect if tag != "sum" else max(1, NB // 4)
+            av.avsa_build_block_mask(q, k, s, n, k_keep, w.blk, flags=flags, out=out, ws=ws)
+            _status_ok(ws)
+            for key, val in out.items():
+                res[f"{tag}.{key}"] = val
+        o, lse = buf(q.shape, torch.bfloat16), buf(q.shape[:3], torch.float32)
+        ws = scratch(av.avsa_sparse_self_attn_workspace_bytes(w.B, w.H, w.n_video, w.d, w.blk))
+        av.avsa_sparse_self_attn(q, k, v, res["tok.col_idx"], res["tok.col_cnt"], w.blk, o=o, lse=lse, ws=ws)
+        _status_ok(ws)
+        res.update(o_base=o.clone(), lse_base=lse.clone())
+        ws = scratch(av.avsa_protected_rows_attn_workspace_bytes(w.B, w.H, w.n_video, w.d, w.blk, n_protect))
+        av.avsa_protected_rows_attn(q, k, v, res["tok.prot_tok"], n_protect, w.blk, o, lse=lse, ws=ws)
+        _status_ok(ws)
+        res.update(o=o, lse=lse)
+        ind = buf((w.B, 8), torch.float32)
+        ws = scratch(av.avsa_cache_indicators_workspace_bytes(w.B, w.n_video, w.n_audio, C))
+        av.avsa_cache_indicators(y_v, yhat_v, y_a, yhat_a, res["tok.prot_tok"], s, s, out=ind, ws=ws)
+        _status_ok(ws)
+        res["indicators"] = ind[:, :6].clone()
+        torch.cuda.synchronize()
+        return res
+
+    a, b = run(0x00), run(0xFF)
+    for key in a:
+        assert torch.equal(a[key].view(torch.uint8), b[key].view(torch.uint8)), f"{key} depends on earlier buffer contents"
