@@ -716,12 +716,27 @@ def test_cache_indicators_match_oracle(Nv, Na, C):
 @pytest.mark.parametrize("B,H,N,d,blk", [(1, 1, 1, 128, 128), (2, 1, 129, 128, 128), (3, 2, 65, 64, 64), (1, 5, 640, 128, 128)])
 def test_degenerate_shapes_whole_path(B, H, N, d, blk):
     """One token, a one-token tail block, several batch items, one head: every call against the oracle."""
-    g = torch.Generator().manual_seed(B * 1000 + N)
-    Na = 7
+    NB = (N + blk - 1) // blk
+    _whole_path_case(B, H, N, d, blk, 7, min(N, 3), max(1, NB // 2), B * 1000 + N)
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_random_shapes_whole_path(seed):
+    """Seeded random batch, heads, lengths (video and audio), tile size, protected count and kept count: every
+    call of the path against the oracle, block-level and token-exact protection."""
+    rng = np.random.default_rng(700 + seed)
+    d = int(rng.choice([64, 128]))
+    B, H = int(rng.integers(1, 3)), int(rng.integers(1, 5))
+    N = int(rng.integers(2, 7 * d))
+    NB = (N + d - 1) // d
+    _whole_path_case(B, H, N, d, d, int(rng.integers(1, 300)), int(rng.integers(0, N // 4 + 2)),
+                     int(rng.integers(1, NB + 1)), 800 + seed)
+
+
+def _whole_path_case(B, H, N, d, blk, Na, n_protect, k_keep, seed):
+    g = torch.Generator().manual_seed(seed)
     q, k, v = (torch.randn((B, H, N, d), generator=g).bfloat16() for _ in range(3))
     qa = torch.randn((B, H, Na, d), generator=g).bfloat16()
-    NB = (N + blk - 1) // blk
-    n_protect, k_keep = min(N, 3), max(1, NB // 2)
     gamma = 1.0 / (H * Na)
     o_a, lse_a, s, ws = av.avsa_cross_attn_scores(qa.cuda(), k.cuda(), v.cuda(), score_gamma=gamma)
     _status_ok(ws)
