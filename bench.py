@@ -55,7 +55,12 @@ def dense_flops(w):
 
 # ------------------------------------------------------------------------------------------------ clocks
 class ClockSampler:
-    """Samples SM clocks and throttle reasons of one GPU with nvidia-smi while the timed region runs."""
+    """Samples SM clock, board power and clock-event reasons of one GPU while the timed region runs.
+
+    Read-only NVML queries from a thread, every few milliseconds; only samples taken between ``begin()`` and
+    ``end()`` (host time stamps taken right before the first launch of the timed region and right after the
+    synchronisation that ends it) enter the summary.  Falls back to an ``nvidia-smi -lms`` child process when the
+    NVML binding is missing."""
 
     FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
@@ -65,8 +70,34 @@ class ClockSampler:
         self.index = index
         self.proc = None
         self.lines = []
+        self.samples = []          # (host time, sm MHz, watts, reason bits)
+        self.nvml = None
+        self.handle = None
+        self.running = False
+        self.t_begin = self.t_end = None
+        self.max_mhz = None
+
+    def _nvml_handle(self):
+        import pynvml
+        pynvml.nvmlInit()
+        self.nvml = pynvml
+        try:
+            pr = torch.cuda.get_device_properties(self.index)
+            bus_id = f"{pr.pci_domain_id:08X}:{pr.pci_bus_id:02X}:{pr.pci_device_id:02X}.0"
+            return pynvml.nvmlDeviceGetHandleByPciBusId(bus_id.encode())
+        except Exception:
+            return pynvml.nvmlDeviceGetHandleByIndex(self.index)
 
     def start(self):
+        try:
+            self.handle = self._nvml_handle()
+            self.max_mhz = float(self.nvml.nvmlDeviceGetMaxClockInfo(self.handle, self.nvml.NVML_CLOCK_SM))
+            self.running = True
+            self.thread = threading.Thread(target=self._poll, daemon=True)
+            self.thread.start()
+            return
+        except Exception:
+            self.handle = None
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
@@ -76,13 +107,48 @@ class ClockSampler:
         except Exception:
             self.proc = None
 
+    def begin(self):
+        self.t_begin = time.perf_counter()
+
+    def end(self):
+        self.t_end = time.perf_counter()
+
+    def _poll(self):
+        n = self.nvml
+        while self.running:
+            try:
+                mhz = n.nvmlDeviceGetClockInfo(self.handle, n.NVML_CLOCK_SM)
+                watts = n.nvmlDeviceGetPowerUsage(self.handle) / 1000.0
+                bits = n.nvmlDeviceGetCurrentClocksEventReasons(self.handle)
+                self.samples.append((time.perf_counter(), float(mhz), watts, int(bits)))
+            except Exception:
+                pass
+            time.sleep(0.002)
+
     def _read(self):
         for line in self.proc.stdout:
             self.lines.append(line.strip())
 
     def stop(self):
+        if self.handle is not None:
+            self.running = False
+            self.thread.join(timeout=2)
+            n = self.nvml
+            inside = [x for x in self.samples
+                      if self.t_begin is not None and self.t_end is not None and self.t_begin <= x[0] <= self.t_end]
+            names = (("hw_slowdown", n.nvmlClocksEventReasonHwSlowdown),
+                     ("hw_thermal_slowdown", n.nvmlClocksEventReasonHwThermalSlowdown),
+                     ("sw_thermal_slowdown", n.nvmlClocksEventReasonSwThermalSlowdown),
+                     ("sw_power_cap", n.nvmlClocksEventReasonSwPowerCap),
+                     ("hw_power_brake_slowdown", n.nvmlClocksEventReasonHwPowerBrakeSlowdown))
+            reasons = sorted({name for _, _, _, bits in inside for name, bit in names if bits & bit})
+            sm = [x[1] for x in inside]
+            return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_min_mhz": min(sm) if sm else None,
+                    "sm_max_mhz": self.max_mhz, "watts_mean": float(np.mean([x[2] for x in inside])) if inside else None,
+                    "samples": len(inside), "source": "nvml, samples inside the timed region only",
+                    "reasons": reasons}
         if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvml and nvidia-smi unavailable"]}
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
@@ -102,7 +168,7 @@ class ClockSampler:
                 if val.lower().startswith("active"):
                     reasons.add(name)
         return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+                "samples": len(sm), "source": "nvidia-smi -lms 100 around the timed region", "reasons": sorted(reasons)}
 
 
 # ------------------------------------------------------------------------------------------------ CPU oracle arm
@@ -216,11 +282,14 @@ def run_ours(args, w):
     sampler = ClockSampler(local_rank) if rank == 0 else None
     if sampler:
         sampler.start()
-        time.sleep(0.3)
+        if sampler.handle is None:
+            time.sleep(0.3)            # the nvidia-smi child needs a moment before its first sample
     # ---- timed region: K whole steps; per-kernel events ride in the same stream
     ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
     start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
+    if sampler:
+        sampler.begin()
     start.record()
     for i in range(args.steps):
         ev[i][0].record()
@@ -232,6 +301,8 @@ def run_ours(args, w):
         ev[i][3].record()
     end.record()
     barrier()
+    if sampler:
+        sampler.end()
     total_ms = start.elapsed_time(end)
     t_cross = float(np.mean([e[0].elapsed_time(e[1]) for e in ev]))
     t_mask = float(np.mean([e[1].elapsed_time(e[2]) for e in ev]))
