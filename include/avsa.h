@@ -224,6 +224,12 @@ AVSA_API int avsa_count_from_percent(int pct, int n);
  * say where the check failed.  For tests and debugging; the hot path never calls it. */
 AVSA_API int avsa_read_status(const void* ws, void* stream, int* detail);
 
+/* Self-test of the device-side time limit (tests only): enqueues one warp that waits on a barrier nothing
+ * ever signals, gives up after `limit_cycles` SM clock cycles (0 .. 2e9, i.e. about a second at most), records
+ * AVSA_ERR_TIMEOUT in the status record at `ws` (>= AVSA_STATUS_BYTES; detail = {99, 0, cycles waited / 1024})
+ * and returns; the context stays usable.  The tile kernels bound every one of their waits the same way. */
+AVSA_API int avsa_selftest_bounded_wait(void* ws, size_t ws_bytes, long long limit_cycles, void* stream);
+
 AVSA_API const char* avsa_status_string(int status);
 AVSA_API int avsa_version(void);
 

@@ -41,7 +41,7 @@ EXPORTS = (
     "avsa_sparse_self_attn", "avsa_sparse_self_attn_workspace_bytes",
     "avsa_protected_rows_attn", "avsa_protected_rows_attn_workspace_bytes",
     "avsa_cache_indicators", "avsa_cache_indicators_workspace_bytes",
-    "avsa_count_from_percent", "avsa_read_status", "avsa_status_string", "avsa_version",
+    "avsa_count_from_percent", "avsa_read_status", "avsa_selftest_bounded_wait", "avsa_status_string", "avsa_version",
 )
 
 
@@ -96,6 +96,8 @@ def load_library() -> ctypes.CDLL:
     lib.avsa_count_from_percent.restype = i
     lib.avsa_read_status.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_int)]
     lib.avsa_read_status.restype = i
+    lib.avsa_selftest_bounded_wait.argtypes = [vp, sz, ctypes.c_longlong, vp]
+    lib.avsa_selftest_bounded_wait.restype = i
     lib.avsa_status_string.argtypes = [i]
     lib.avsa_status_string.restype = ctypes.c_char_p
     lib.avsa_version.argtypes = []
@@ -163,6 +165,12 @@ def avsa_read_status(ws: torch.Tensor) -> Tuple[int, Tuple[int, int, int]]:
 # ------------------------------------------------------------------------------------------------
 # the three calls
 # ------------------------------------------------------------------------------------------------
+def avsa_selftest_bounded_wait(ws: torch.Tensor, limit_cycles: int) -> None:
+    """Enqueues the wait that nothing ends; read the outcome with avsa_read_status(ws)."""
+    st = load_library().avsa_selftest_bounded_wait(_ptr(ws), ws.numel(), int(limit_cycles), _stream(ws.device))
+    _check(st, "avsa_selftest_bounded_wait")
+
+
 def avsa_cross_attn_scores_workspace_bytes(B, H, Nq, Nk, d) -> int:
     return int(load_library().avsa_cross_attn_scores_workspace_bytes(B, H, Nq, Nk, d))
 

@@ -59,6 +59,38 @@ __global__ void __launch_bounds__(1024) prep_sparse_kernel(StatusRecord* st, con
   }
 }
 
+// Self-test of the time-limited wait used throughout the tile kernels: one warp waits on an mbarrier that nothing
+// ever arrives on, gives up after `limit_cycles`, records AVSA_ERR_TIMEOUT in the status record and returns.
+constexpr int kWhereSelfTestWait = 99;
+__global__ void __launch_bounds__(32) bounded_wait_selftest_kernel(StatusRecord* st, long long limit_cycles) {
+  __shared__ __align__(8) uint64_t bar;
+  const uint32_t b = smem_u32(&bar);
+  if (threadIdx.x == 0) {
+    st->code = 0;
+    st->where = 0;
+    st->item = 0;
+    st->aux = 0;
+    st->redo_count = 0;
+    st->next_item = 0;
+    mbar_init(b, 1);
+    fence_mbar_init();
+  }
+  __syncwarp();
+  bool done = false;
+  if (threadIdx.x == 0) {
+    const long long t0 = clock64();
+    while (!(done = mbar_try_wait(b, 0))) {
+      const long long waited = clock64() - t0;
+      if (waited > limit_cycles) {
+        report_status(st, AVSA_ERR_TIMEOUT, kWhereSelfTestWait, 0, static_cast<int>(min(waited >> 10, 0x7fffffffll)));
+        break;
+      }
+    }
+  }
+  __syncwarp();
+  if (threadIdx.x == 0) mbar_inval(b);
+}
+
 template <int BLK, int D>
 static int launch_sparse_attn(int B, int H, int N, const avsa_bf16_4d& q, const avsa_bf16_4d& k,
                               const avsa_bf16_4d& v, void* o, const AttnParams& prm, int* redo, cudaStream_t st) {
@@ -96,6 +128,14 @@ extern "C" __attribute__((visibility("default"))) void avsa_debug_set_trace(long
   g_trace_buffer = device_buffer;
 }
 #endif
+
+extern "C" int avsa_selftest_bounded_wait(void* ws, size_t ws_bytes, long long limit_cycles, void* stream) {
+  if (ws == nullptr || ws_bytes < kStatusBytes) return AVSA_ERR_WORKSPACE;
+  if (limit_cycles < 0 || limit_cycles > 2000000000ll) return AVSA_ERR_INVALID_ARG;     // about a second at most
+  if (!device_is_sm100()) return AVSA_ERR_UNSUPPORTED;
+  bounded_wait_selftest_kernel<<<1, 32, 0, as_stream(stream)>>>(static_cast<StatusRecord*>(ws), limit_cycles);
+  return cudaGetLastError() == cudaSuccess ? AVSA_OK : AVSA_ERR_CUDA;
+}
 
 extern "C" size_t avsa_sparse_self_attn_workspace_bytes(int B, int H, int N, int d, int blk) {
   if (B <= 0 || H <= 0 || N <= 0 || d <= 0 || blk <= 0) return 0;

@@ -871,3 +871,23 @@ def test_results_do_not_depend_on_what_the_buffers_held_before(name):
     a, b = run(0x00), run(0xFF)
     for key in a:
         assert torch.equal(a[key].view(torch.uint8), b[key].view(torch.uint8)), f"{key} depends on earlier buffer contents"
+
+
+# ------------------------------------------------------------------------------------------- time-limited waits
+def test_a_wait_that_nothing_ends_times_out_and_leaves_the_context_usable():
+    """Every wait inside the tile kernels is time-limited.  The self-test kernel waits on a barrier that nothing
+    signals: it must give up after the limit, report AVSA_ERR_TIMEOUT through the status record, and the next
+    ordinary call on the same context must work."""
+    ws = torch.empty(av.AVSA_STATUS_BYTES, dtype=torch.uint8, device="cuda")
+    limit = 2_000_000                                           # about a millisecond
+    av.avsa_selftest_bounded_wait(ws, limit)
+    code, (where, item, waited_k) = av.avsa_read_status(ws)
+    assert code == av.AVSA_ERR_TIMEOUT and where == 99 and item == 0
+    assert limit // 1024 <= waited_k <= 4 * limit // 1024
+    assert "timed out" in av.status_string(code)
+    with pytest.raises(av.AvsaError):
+        av.avsa_selftest_bounded_wait(ws, 3_000_000_000)        # limits beyond about a second are refused
+    w = wl.WORKLOADS["tiny"]
+    NB = w.n_blocks
+    idx = np.broadcast_to(np.arange(NB, dtype=np.int32), (w.B, w.H, NB, NB)).copy()
+    _run_sparse_case(w, 1, idx, np.full((w.B, w.H, NB), NB, np.int32))
