@@ -76,10 +76,9 @@ __global__ void __launch_bounds__(32) bounded_wait_selftest_kernel(StatusRecord*
     fence_mbar_init();
   }
   __syncwarp();
-  bool done = false;
   if (threadIdx.x == 0) {
     const long long t0 = clock64();
-    while (!(done = mbar_try_wait(b, 0))) {
+    while (!mbar_try_wait(b, 0)) {
       const long long waited = clock64() - t0;
       if (waited > limit_cycles) {
         report_status(st, AVSA_ERR_TIMEOUT, kWhereSelfTestWait, 0, static_cast<int>(min(waited >> 10, 0x7fffffffll)));
