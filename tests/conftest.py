@@ -24,3 +24,14 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+def pytest_terminal_summary(terminalreporter):
+    """Largest errors the parity helpers saw (against the bars in parity_bars.py)."""
+    try:
+        import parity_bars
+    except Exception:
+        return
+    if any(v > 0 for v in parity_bars.WORST.values()):
+        terminalreporter.write_line("largest parity errors of this session: " +
+                                    ", ".join(f"{k} {v:.3e}" for k, v in parity_bars.WORST.items()))
