@@ -546,6 +546,51 @@ def time_layer_step(av, w, seed, dev, n_iter=3, token_exact=False):
             "protected_blocks": int(m["prot_blk"].sum().item()), "n_blocks": NB}
 
 
+def run_single_call(args, w):
+    """Times ONE call of the path alone on the chosen workload (its inputs come from the other calls, run once
+    before): ``--call cross | cross_rev | mask | attn | rows``.  This is also the command the per-call ncu
+    captures under profiles/ run, since it launches little besides the kernels of that call."""
+    from paper_2608_15522_b200 import binding as av
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    q, k, v = wl.make_self_qkv(w, 0, dev)
+    qa, kc, vc = wl.make_cross_qkv(w, 0, dev)
+    n_protect = av.avsa_count_from_percent(w.protect_pct, w.n_video)
+    k_keep = max(1, av.avsa_count_from_percent(w.keep_pct, w.n_blocks))
+    gamma = 1.0 / (w.H * w.n_audio)
+    o_a, lse, s, ws1 = av.avsa_cross_attn_scores(qa, kc, vc, score_gamma=gamma)
+    flags = av.AVSA_PROTECT_TOKENS if args.call == "rows" else av.AVSA_PROTECT_ROWS
+    m = av.avsa_build_block_mask(q, k, s, n_protect, k_keep, w.blk, flags=flags)
+    o, _, ws3 = av.avsa_sparse_self_attn(q, k, v, m["col_idx"], m["col_cnt"], w.blk)
+    if args.call == "cross":
+        fn = lambda: av.avsa_cross_attn_scores(qa, kc, vc, scores=s, score_gamma=gamma, o=o_a, lse=lse, ws=ws1)
+    elif args.call == "cross_rev":
+        o_r, lse_r, s_r, ws_r = av.avsa_cross_attn_scores(kc, qa, qa, score_gamma=1.0 / (w.H * w.n_video))
+        fn = lambda: av.avsa_cross_attn_scores(kc, qa, qa, scores=s_r, score_gamma=1.0 / (w.H * w.n_video), o=o_r,
+                                               lse=lse_r, ws=ws_r)
+    elif args.call == "mask":
+        fn = lambda: av.avsa_build_block_mask(q, k, s, n_protect, k_keep, w.blk, flags=flags, out=m, ws=m["ws"])
+    elif args.call == "attn":
+        fn = lambda: av.avsa_sparse_self_attn(q, k, v, m["col_idx"], m["col_cnt"], w.blk, o=o, ws=ws3)
+    else:
+        ws4 = av.avsa_protected_rows_attn(q, k, v, m["prot_tok"], n_protect, w.blk, o)
+        fn = lambda: av.avsa_protected_rows_attn(q, k, v, m["prot_tok"], n_protect, w.blk, o, ws=ws4)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    for _ in range(max(args.warmup, 1)):
+        fn()
+    times = []
+    for _ in range(args.steps):
+        flush.fill_(1)                     # write a buffer larger than L2 between timed launches
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        fn()
+        b.record()
+        torch.cuda.synchronize()
+        times.append(a.elapsed_time(b))
+    print(json.dumps({"call": args.call, "workload": w.name, "steps": args.steps, "ms_median": float(np.median(times)),
+                      "ms_min": float(np.min(times)), "l2": "256 MB written between timed launches"}))
+
+
 def run_sweep(args, w):
     """Keep ratio x protected fraction grid on one workload (the mid-length sweep of the benchmark plan)."""
     from paper_2608_15522_b200 import binding as av
@@ -654,6 +699,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--keep-pct", type=int, default=None)
     ap.add_argument("--protect-pct", type=int, default=None)
+    ap.add_argument("--call", default=None, choices=["cross", "cross_rev", "mask", "attn", "rows"],
+                    help="time one call of the path alone (L2 flushed between launches)")
     ap.add_argument("--sweep", action="store_true", help="keep x protect grid on the chosen workload (one JSON line)")
     ap.add_argument("--loop", action="store_true", help="multi-step denoising loop on the chosen workload")
     ap.add_argument("--loop-steps", type=int, default=8)
@@ -666,7 +713,9 @@ def main():
     if args.keep_pct is not None or args.protect_pct is not None:
         w = w.with_ratios(args.keep_pct if args.keep_pct is not None else w.keep_pct,
                           args.protect_pct if args.protect_pct is not None else w.protect_pct)
-    if args.sweep:
+    if args.call:
+        run_single_call(args, w)
+    elif args.sweep:
         run_sweep(args, w)
     elif args.loop and args.lag > 0:
         run_loop_lagged(args, w)

@@ -19,9 +19,11 @@
  *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  No call reads device
  *     data on the host, so the calls may be recorded into a CUDA graph by stream capture (not on the legacy
  *     default stream) and replayed; pointers, sizes and counts are fixed at capture time.
- *   - `ws` is scratch of at least the matching *_workspace_bytes(); its first 16 bytes are a status
- *     record the kernels fill when a device-side check fails (a wait that ran out of time, or a
- *     malformed column list).  Calls on the same workspace must not overlap on the GPU.
+ *   - `ws` is scratch of at least the matching *_workspace_bytes().  Its first AVSA_STATUS_BYTES (256) bytes
+ *     are reserved for a 24-byte status record of six int32: code (avsa_status), where, item, aux -- filled
+ *     when a device-side check fails (a wait that ran out of time, or a malformed column list) -- then at
+ *     byte 16 the count of recomputed work items (see below) and at byte 20 the head of the persistent
+ *     kernels' work queue.  Calls on the same workspace must not overlap on the GPU.
  *   - The attention calls (cross-attention pass 1, sparse self-attention, protected rows) run a kernel that
  *     normalises each row by the maximum of its first key tile instead of a running maximum (softmax is
  *     invariant to that shift), and behind it an exact-rescaling kernel for the work items whose rows
@@ -98,8 +100,9 @@ typedef struct {
  * accumulates layers; score_beta = alpha with score_gamma = (1-alpha)/(H*Nq) is Eq. 4.
  * With score_beta == 0 the previous contents of scores are ignored (may be uninitialised).
  * o, lse and scores may each be NULL to skip that output (scores == NULL skips the second pass).
- * softmax_scale == 0 means 1/sqrt(d).  Nq <= 512 when scores are requested (any Nq otherwise, which serves the
- * reverse, video->audio direction of the bidirectional pair).  The head sum is taken in a fixed order, so
+ * softmax_scale == 0 means 1/sqrt(d).  When scores are requested min(Nq, Nk) <= 512 (the score pass keeps the
+ * shorter axis of a head on chip: the audio queries, or, in the reverse video->audio direction of the
+ * bidirectional pair, the audio keys); without scores any Nq and Nk.  The head sum is taken in a fixed order, so
  * results reproduce bit for bit.  `o` has strides (o_stride_b, o_stride_h, o_stride_n) = q's.
  */
 AVSA_API int avsa_cross_attn_scores(int B, int H, int Nq, int Nk, int d, avsa_bf16_4d q, avsa_bf16_4d k, avsa_bf16_4d v,
@@ -209,6 +212,8 @@ AVSA_API size_t avsa_cache_indicators_workspace_bytes(int B, int Nv, int Na, int
  *     on the GPU (different streams) race on the array: serialise them.
  *   - The mask kernels have no device-side failure mode (no waits, no list input), so there is no
  *     status record to read after this call.
+ *   - Call it from one host thread at a time per device.  The looked-up address belongs to the current
+ *     context: after cudaDeviceReset() it is stale, and the library must be reloaded before the next call.
  */
 #define AVSA_STATIC_SCRATCH_BYTES (16u << 20)
 AVSA_API int avsa_build_block_mask_static(int B, int H, int N, int d, int blk, avsa_bf16_4d q, avsa_bf16_4d k,

@@ -249,7 +249,7 @@ def avsa_build_block_mask_static(q, k, scores, n_protect, k_keep, blk, out, flag
     """avsa_build_block_mask without a workspace: the library's built-in scratch array is used.
 
     For callers that must not allocate.  Accordingly this wrapper allocates nothing either: every output
-    tensor (block_scores, col_idx, col_cnt, prot_tok, prot_blk) must be supplied in ``out``.  Shapes that
+    tensor (block_scores, col_idx, col_cnt, and prot_tok / prot_blk if wanted) must be supplied in ``out``.  Shapes that
     need more scratch than AVSA_STATIC_SCRATCH_BYTES raise AvsaError(AVSA_ERR_WORKSPACE).  The first call
     on a device resolves the array's address; make it before any stream capture.  Calls share the array, so
     do not let two of them overlap on the GPU.
@@ -258,8 +258,8 @@ def avsa_build_block_mask_static(q, k, scores, n_protect, k_keep, blk, out, flag
     B, H, N, d = q.shape
     st = lib.avsa_build_block_mask_static(B, H, N, d, blk, _t4(q), _t4(k), _ptr(scores), int(n_protect), int(k_keep),
                                           int(flags), float(softmax_scale), _ptr(out["block_scores"]),
-                                          _ptr(out["col_idx"]), _ptr(out["col_cnt"]), _ptr(out["prot_tok"]),
-                                          _ptr(out["prot_blk"]), _stream(q.device))
+                                          _ptr(out["col_idx"]), _ptr(out["col_cnt"]), _ptr(out.get("prot_tok")),
+                                          _ptr(out.get("prot_blk")), _stream(q.device))
     _check(st, "avsa_build_block_mask_static")
     return out
 

@@ -63,20 +63,7 @@ struct AttnParams {
   int Nq, NQT;              // query rows and query tiles
   int Nk, NKB;              // key rows and key tiles
   float scale_log2;         // softmax_scale * log2(e)
-#ifdef AVSA_TRACE
-  long long* trace;         // [3 roles][64 tiles][8 stamps] clock64 stamps of CTA (0,0,0), for pipeline analysis
-#endif
 };
-
-#ifdef AVSA_TRACE
-#define AVSA_STAMP(role, tile, slot)                                                                    \
-  do {                                                                                                  \
-    if (p.trace != nullptr && blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && (tile) < 64)     \
-      p.trace[((role) * 64 + (tile)) * 8 + (slot)] = clock64();                                         \
-  } while (0)
-#else
-#define AVSA_STAMP(role, tile, slot) do { } while (0)
-#endif
 
 // One work item of the tile kernel: query tile `bx` (MODE_LIST) or query tile / key split `bx`
 // (range modes) of head `by`, batch item `bz`.  Called once per flagged work item by attn_redo_kernel;
@@ -252,7 +239,6 @@ __device__ __forceinline__ void attn_fwd_body(const CUtensorMap* tmq, const CUte
           const uint32_t k_lo = k_lo0 + sk * (L::kTileBytes >> 4);
           const uint32_t tm_s = tmem_u + (w << 7);
           if (leader) {
-            AVSA_STAMP(0, t, 0);
 #pragma unroll
             for (int ks = 0; ks < D / 16; ks++) {
               const uint32_t qoff = ((ks >> 2) * QPANEL_BYTES + (ks & 3) * 32) >> 4;
@@ -261,7 +247,6 @@ __device__ __forceinline__ void attn_fwd_body(const CUtensorMap* tmq, const CUte
             }
             umma_commit(BAR(S_FULL + w));
             umma_commit(BAR(K_EMPTY + sk));
-            AVSA_STAMP(0, t, 1);
           }
           __syncwarp();
           if (++sk == kStages) { sk = 0; fk ^= 1; }
@@ -280,7 +265,6 @@ __device__ __forceinline__ void attn_fwd_body(const CUtensorMap* tmq, const CUte
           const int u = t - 1, w = u & 1, i = u >> 1;
           // P arrives in two halves of the key axis: the first half of the product starts while the
           // softmax group is still exponentiating the second half
-          if (leader) AVSA_STAMP(0, u, 2);
           ok = wait_all(P_FULL + 2 * w, i & 1, kWherePFull, u);
           if (!ok) break;
           tc_fence_after();
@@ -288,7 +272,6 @@ __device__ __forceinline__ void attn_fwd_body(const CUtensorMap* tmq, const CUte
           const uint32_t tm_p = tmem_u + (w << 7), tm_o = tmem_u + 256u + (w << 7);
           const uint32_t acc0 = i > 0 ? 1u : 0u;
           if (leader) {
-            AVSA_STAMP(0, u, 3);
 #pragma unroll
             for (int ks = 0; ks < BLK / 32; ks++)
               umma_ts(tm_o, tm_p + ks * 8, desc64(v_lo + ks * (2048 >> 4)), idesc_pv, ks > 0 ? 1u : acc0);
@@ -302,7 +285,6 @@ __device__ __forceinline__ void attn_fwd_body(const CUtensorMap* tmq, const CUte
             for (int ks = BLK / 32; ks < BLK / 16; ks++)
               umma_ts(tm_o, tm_p + ks * 8, desc64(v_lo + ks * (2048 >> 4)), idesc_pv, 1u);
             umma_commit(BAR(V_EMPTY + sv));
-            AVSA_STAMP(0, u, 4);
           }
           __syncwarp();
           if (++sv == kStages) { sv = 0; fv ^= 1; }
@@ -326,17 +308,14 @@ __device__ __forceinline__ void attn_fwd_body(const CUtensorMap* tmq, const CUte
     bool ok = true;
     for (int i = 0; i < nw && ok; i++) {
       const int t = 2 * i + w;
-      if ((warp & 3) == 0 && lane == 0) AVSA_STAMP(1 + w, t, 0);
       ok = wait_or_abort(S_FULL + w, i & 1, kWhereSFull, t);
       if (!ok) break;
       tc_fence_after();
-      if ((warp & 3) == 0 && lane == 0) AVSA_STAMP(1 + w, t, 1);
       uint32_t s[BLK];
 #pragma unroll
       for (int c = 0; c < BLK / 32; c++)
         tmem_ld32(TM_S[w] + lane_off + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
       tmem_wait_ld();
-      if ((warp & 3) == 0 && lane == 0) AVSA_STAMP(1 + w, t, 2);
       if (t == cnt - 1 && ragged_valid < BLK) {
 #pragma unroll
         for (int j = 0; j < BLK; j++)
@@ -372,7 +351,6 @@ __device__ __forceinline__ void attn_fwd_body(const CUtensorMap* tmq, const CUte
         }
       }
       l_run *= factor;
-      if ((warp & 3) == 0 && lane == 0) AVSA_STAMP(1 + w, t, 3);
       // p = exp2(s * c - m) on pairs: one packed FMA, two EX2, one packed add, one bf16x2 convert per pair
       const uint64_t c2 = pack_f32x2(p.scale_log2, p.scale_log2);
       const uint64_t nm2 = pack_f32x2(-m_run, -m_run);
@@ -400,11 +378,9 @@ __device__ __forceinline__ void attn_fwd_body(const CUtensorMap* tmq, const CUte
       unpack_f32x2(add_f32x2(add_f32x2(sum2[0], sum2[1]), add_f32x2(sum2[2], sum2[3])), sa, sb);
       const float sum = sa + sb;
       l_run += sum;
-      if ((warp & 3) == 0 && lane == 0) AVSA_STAMP(1 + w, t, 4);
       tmem_wait_st();
       tc_fence_before();
       mbar_arrive(BAR(P_FULL + 2 * w + 1));
-      if ((warp & 3) == 0 && lane == 0) AVSA_STAMP(1 + w, t, 5);
     }
     // publish this group's statistics, then merge the two halves of the key axis
     stats[(w * 2 + 0) * 128 + row] = m_run;

@@ -55,7 +55,7 @@ struct PersistSmem {
   static constexpr int kBars = kStage + kQBytes;
   static constexpr int kNumBars = 2 * kPQB + 2 * kPKS + 2 * kPVS + 18 + 2 * kPRing;
   static constexpr int kStats = kBars + kNumBars * 8;          // float mref[128], lsum[2][128]
-  static constexpr int kItems = kStats + 3 * 128 * 4;          // int {item, cnt}[kPRing], redo flag
+  static constexpr int kItems = kStats + 3 * 128 * 4;          // int {item, cnt}[kPRing], two redo flags
   static constexpr int kMisc = kItems + 8 * kPRing + 16;       // tmem base, stop flag
   static constexpr int kTotal = kMisc + 16;
 };
@@ -129,7 +129,10 @@ attn_persist_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_consta
   constexpr int NCH = BLK / 32;
   float* mref_s = reinterpret_cast<float*>(smem + L::kStats);
   float* lsum_s = mref_s + 128;                                              // [2][128]
-  volatile int* items = reinterpret_cast<volatile int*>(smem + L::kItems);   // {item, cnt} x kPRing, then the redo flag
+  volatile int* items = reinterpret_cast<volatile int*>(smem + L::kItems);   // {item, cnt} x kPRing, then two redo flags
+  // One redo flag per item parity: the flag of item n is cleared after item n's second row-sum barrier, and the
+  // first thread that can set the flag of item n + 2 has passed that barrier itself, so a set never meets a
+  // pending clear (with a single flag, a fast warp of the other group could set it for item n + 1 first).
   constexpr int REDO = 2 * kPRing;
   volatile uint32_t* misc = reinterpret_cast<volatile uint32_t*>(smem + L::kMisc);   // [0] tmem base, [1] stop
 
@@ -167,6 +170,7 @@ attn_persist_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_consta
     mbar_init(BAR(STAGE_FULL), 256);
     misc[1] = 0u;
     items[REDO] = 0;
+    items[REDO + 1] = 0;
     fence_mbar_init();
     prefetch_tmap(&tmq);
     prefetch_tmap(&tmk);
@@ -579,7 +583,7 @@ attn_persist_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_consta
       // A row sum beyond 2^64 (or not finite) means the row outgrew its first-tile reference: the item is left
       // to the exact-rescaling kernel.  (With 64-row tiles the upper 64 lanes hold no rows: the 128-row MMA filled
       // them from whatever follows the Q tile in shared memory, and their sums mean nothing.)
-      if (row < BLK && !(l_run <= kFastRowSumLimit)) items[REDO] = 1;
+      if (row < BLK && !(l_run <= kFastRowSumLimit)) items[REDO + (n & 1)] = 1;
       lsum_s[w * 128 + row] = l_run;
       // the staged output tile of the item before must have been read by its TMA store before anybody writes the
       // staging buffer again; the thread that issued the store makes sure of it before it joins the barrier below
@@ -589,12 +593,12 @@ attn_persist_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_consta
       ok = __all_sync(FULLM, wait_or_stop(LSUM_A, n & 1, kPersistLsum, n));
       if (!ok) break;
       const float Lsum = l_run + lsum_s[(1 - w) * 128 + row];
-      const bool redo = items[REDO] != 0;
+      const bool redo = items[REDO + (n & 1)] != 0;
       mbar_arrive(BAR(LSUM_B));                           // everyone has read the sums and the flag
       ok = __all_sync(FULLM, wait_or_stop(LSUM_B, n & 1, kPersistLsum, n));
       if (!ok) break;
       if (tid == 128) {
-        items[REDO] = 0;
+        items[REDO + (n & 1)] = 0;
         if (redo) redo_list[atomicAdd(&p.status->redo_count, 1)] = item;
       }
       ok = __all_sync(FULLM, wait_or_stop(O_FULL, n & 1, kPersistOFull, n));

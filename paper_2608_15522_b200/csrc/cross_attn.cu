@@ -434,10 +434,10 @@ static CrossPlan make_cross_plan(int B, int H, int Nq, int Nk, int d) {
   c.blk = d;   // (blk, d) = (128,128) or (64,64)
   c.NQT = (Nq + c.blk - 1) / c.blk;
   c.NKB = (Nk + c.blk - 1) / c.blk;
-  // One work item per SM (148 SMs, one CTA each): a single wave.  Two items per SM were measured slower on the
+  // One work item per SM (one CTA each): a single wave.  Two items per SM were measured slower on the
   // Ovi-class shape (210 vs 196 us for the call): every item pays its own pipeline fill, partial-result
   // write-out and merge work.
-  const int target = 148;
+  const int target = persistent_grid(1 << 30);
   int want_split = target / (B * H * c.NQT);
   if (want_split < 1) want_split = 1;
   if (want_split > c.NKB) want_split = c.NKB;

@@ -83,11 +83,9 @@ __global__ void __launch_bounds__(256) pool_kernel(const __nv_bfloat16* __restri
 }
 
 // ------------------------------------------------------------------------------------------------
-// (ii) block scores Bs[bh, i, j] = qbar[bh,i,:] . kbar[bh,j,:] * scale.  The pooled means are fp32 and the
-// scores feed a top-k, so the product keeps fp32 accuracy: every operand is split into two tf32 halves
-// (x = hi + lo exactly to 2^-22) and three tensor-core products a_lo*b_hi + a_hi*b_lo + a_hi*b_hi are
-// accumulated in fp32 (warp-level m16n8k8 MMAs; the problem is far too small for the tcgen05 path).
-// 64x64 tile per CTA, 4 warps x (32x32), both operand tiles staged row-major in shared memory.
+// fp32-accurate products on the warp-level tensor cores: every operand is split into two tf32 halves
+// (x = hi + lo exactly to 2^-22) and three products a_lo*b_hi + a_hi*b_lo + a_hi*b_hi are accumulated in
+// fp32 (m16n8k8 MMAs; the block-score problem is far too small for the tcgen05 path).
 // ------------------------------------------------------------------------------------------------
 __device__ __forceinline__ void split_tf32(float x, uint32_t& hi, uint32_t& lo) {
   asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(hi) : "f"(x));
@@ -99,90 +97,6 @@ __device__ __forceinline__ void mma_tf32(float (&d)[4], const uint32_t (&a)[4], 
       "mma.sync.aligned.m16n8k8.row.col.f32.tf32.tf32.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
       : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b[0]), "r"(b[1]));
-}
-
-template <int D>
-__global__ void __launch_bounds__(128) block_score_kernel(const float* __restrict__ qbar,
-                                                          const float* __restrict__ kbar, float* __restrict__ bs,
-                                                          int NB, float scale) {
-  constexpr int PITCH = D + 4;     // floats; keeps 16-byte alignment and makes fragment loads conflict-free
-  extern __shared__ __align__(16) float score_smem[];
-  float* sq = score_smem;
-  float* sk = score_smem + 64 * PITCH;
-  // Staged behind the pooling grid (programmatic dependent launch) and waits for it here; the pooling grid
-  // in turn retires only after the token select, so the list kernel behind this one, which waits for this
-  // grid, sees the block flags too.
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  asm volatile("griddepcontrol.wait;" ::: "memory");
-  const int bh = blockIdx.z, i0 = blockIdx.y * 64, j0 = blockIdx.x * 64;
-  const float* qb = qbar + static_cast<int64_t>(bh) * NB * D;
-  const float* kb = kbar + static_cast<int64_t>(bh) * NB * D;
-  // both 64 x D tiles go straight from global to shared memory, every 16-byte piece in flight at once
-  // (rows beyond NB are zero-filled by a zero source size)
-#pragma unroll
-  for (int it = 0; it < 64 * (D / 4) / 128; it++) {
-    const int e = it * 128 + threadIdx.x;
-    const int r = e / (D / 4), c4 = e % (D / 4);
-    const bool qv = (i0 + r < NB), kv = (j0 + r < NB);
-    const float* gq = qb + static_cast<int64_t>(qv ? i0 + r : 0) * D + c4 * 4;
-    const float* gk = kb + static_cast<int64_t>(kv ? j0 + r : 0) * D + c4 * 4;
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(static_cast<uint32_t>(
-                     __cvta_generic_to_shared(sq + r * PITCH + c4 * 4))), "l"(gq), "r"(qv ? 16 : 0) : "memory");
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(static_cast<uint32_t>(
-                     __cvta_generic_to_shared(sk + r * PITCH + c4 * 4))), "l"(gk), "r"(kv ? 16 : 0) : "memory");
-  }
-  asm volatile("cp.async.wait_all;" ::: "memory");
-  __syncthreads();
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int g = lane >> 2, t = lane & 3;
-  const int wr = (warp >> 1) * 32, wc = (warp & 1) * 32;     // this warp's 32x32 corner inside the tile
-  float acc[2][4][4];
-#pragma unroll
-  for (int mi = 0; mi < 2; mi++)
-#pragma unroll
-    for (int ni = 0; ni < 4; ni++)
-#pragma unroll
-      for (int r = 0; r < 4; r++) acc[mi][ni][r] = 0.f;
-#pragma unroll 2
-  for (int k0 = 0; k0 < D; k0 += 8) {
-    uint32_t ah[2][4], al[2][4], bhh[4][2], bl[4][2];
-#pragma unroll
-    for (int mi = 0; mi < 2; mi++) {
-      const float* base = sq + (wr + mi * 16 + g) * PITCH + k0 + t;
-      split_tf32(base[0], ah[mi][0], al[mi][0]);
-      split_tf32(base[8 * PITCH], ah[mi][1], al[mi][1]);
-      split_tf32(base[4], ah[mi][2], al[mi][2]);
-      split_tf32(base[8 * PITCH + 4], ah[mi][3], al[mi][3]);
-    }
-#pragma unroll
-    for (int ni = 0; ni < 4; ni++) {
-      const float* base = sk + (wc + ni * 8 + g) * PITCH + k0 + t;
-      split_tf32(base[0], bhh[ni][0], bl[ni][0]);
-      split_tf32(base[4], bhh[ni][1], bl[ni][1]);
-    }
-#pragma unroll
-    for (int mi = 0; mi < 2; mi++)
-#pragma unroll
-      for (int ni = 0; ni < 4; ni++) {
-        mma_tf32(acc[mi][ni], al[mi], bhh[ni]);     // small terms first
-        mma_tf32(acc[mi][ni], ah[mi], bl[ni]);
-        mma_tf32(acc[mi][ni], ah[mi], bhh[ni]);
-      }
-  }
-#pragma unroll
-  for (int mi = 0; mi < 2; mi++)
-#pragma unroll
-    for (int half = 0; half < 2; half++) {
-      const int i = i0 + wr + mi * 16 + g + half * 8;
-      if (i >= NB) continue;
-#pragma unroll
-      for (int ni = 0; ni < 4; ni++) {
-        const int j = j0 + wc + ni * 8 + 2 * t;
-        float* dst = bs + (static_cast<int64_t>(bh) * NB + i) * NB + j;
-        if (j < NB) dst[0] = acc[mi][ni][half * 2] * scale;
-        if (j + 1 < NB) dst[1] = acc[mi][ni][half * 2 + 1] * scale;
-      }
-    }
 }
 
 // Adds one warp's digits to a shared-memory histogram.  When every participating lane holds the same
@@ -350,30 +264,17 @@ __global__ void __launch_bounds__(1024) token_select_kernel(const float* __restr
 
 // ------------------------------------------------------------------------------------------------
 // (iv) per-(head, query block) top-k_keep of a block-score row, protection OR (Eq. 9), ascending
-// list emission.  One warp per row, 4 rows per CTA; the row's keys live in registers (KPL per lane,
-// element j*32+lane in slot j).  The radix select stops as soon as the bin that holds the k-th key
-// is taken whole.
+// list emission.  One warp per row; the row's keys live in registers (KPL per lane, element j*32+lane
+// in slot j).  The radix select stops as soon as the bin that holds the k-th key is taken whole.
+// `src` is the row of block scores (global or shared memory), `bins` 256 ints of shared memory owned
+// by this warp.
 // ------------------------------------------------------------------------------------------------
 template <int KPL>
-__global__ void __launch_bounds__(128) row_select_kernel(const float* __restrict__ bs, const uint8_t* __restrict__ prot_blk,
-                                                         int H, int NB, int k_keep, int protect_rows,
-                                                         int protect_cols, int total_rows, int32_t* __restrict__ col_idx,
-                                                         int32_t* __restrict__ col_cnt) {
-  __shared__ int all_bins[4][256];
-  asm volatile("griddepcontrol.wait;" ::: "memory");   // block scores and block flags come from earlier kernels
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  int* bins = all_bins[warp];
-  const int row = blockIdx.x * 4 + warp;      // row = (b*H + h)*NB + qb
-  if (row >= total_rows) return;
-  const int qb = row % NB;
-  const int b = row / (NB * H);
-  const float* src = bs + static_cast<int64_t>(row) * NB;
-  int32_t* out = col_idx + static_cast<int64_t>(row) * NB;
-  const uint8_t* pb = prot_blk + static_cast<int64_t>(b) * NB;
-  const bool row_prot = protect_rows && pb[qb] != 0;
+__device__ __forceinline__ void select_row(const float* src, const uint8_t* __restrict__ pb, bool row_prot, int NB,
+                                           int k_keep, int protect_cols, int* bins, int lane,
+                                           int32_t* __restrict__ out, int32_t* __restrict__ cnt_out) {
   const unsigned lt = (1u << lane) - 1u;
   const bool keep_all = row_prot || k_keep >= NB;
-
   uint32_t keys[KPL];
   uint32_t T = 0;
   int want = 0;
@@ -381,7 +282,7 @@ __global__ void __launch_bounds__(128) row_select_kernel(const float* __restrict
 #pragma unroll
     for (int j = 0; j < KPL; j++) {
       const int i = j * 32 + lane;
-      keys[j] = (i < NB) ? rank_key(__ldg(src + i)) : 0u;
+      keys[j] = (i < NB) ? rank_key(src[i]) : 0u;
     }
     uint32_t prefix = 0, mask = 0;
     want = k_keep;
@@ -447,7 +348,144 @@ __global__ void __launch_bounds__(128) row_select_kernel(const float* __restrict
     pos += __popc(km);
   }
   for (int i = pos + lane; i < NB; i += 32) out[i] = -1;
-  if (lane == 0) col_cnt[row] = pos;
+  if (lane == 0) *cnt_out = pos;
+}
+
+// Lists from a block-score tensor that is already in global memory (AVSA_USE_GIVEN_BLOCK_SCORES): one warp
+// per row, 4 rows per CTA.
+template <int KPL>
+__global__ void __launch_bounds__(128) row_select_kernel(const float* __restrict__ bs, const uint8_t* __restrict__ prot_blk,
+                                                         int H, int NB, int k_keep, int protect_rows,
+                                                         int protect_cols, int total_rows, int32_t* __restrict__ col_idx,
+                                                         int32_t* __restrict__ col_cnt) {
+  __shared__ int all_bins[4][256];
+  asm volatile("griddepcontrol.wait;" ::: "memory");   // the block flags come from the kernel before
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int row = blockIdx.x * 4 + warp;      // row = (b*H + h)*NB + qb
+  if (row >= total_rows) return;
+  const int qb = row % NB;
+  const int b = row / (NB * H);
+  const uint8_t* pb = prot_blk + static_cast<int64_t>(b) * NB;
+  select_row<KPL>(bs + static_cast<int64_t>(row) * NB, pb, protect_rows && pb[qb] != 0, NB, k_keep, protect_cols,
+                  all_bins[warp], lane, col_idx + static_cast<int64_t>(row) * NB, col_cnt + row);
+}
+
+// ------------------------------------------------------------------------------------------------
+// (ii)+(iv) fused: block scores Bs[bh, i, j] = qbar[bh,i,:] . kbar[bh,j,:] * scale for a strip of 16 query
+// blocks against every key block, kept in shared memory, then the lists of those 16 rows straight from
+// there.  One CTA of 8 warps per strip: each warp computes 32-column chunks of the strip with 3xTF32
+// m16n8k8 MMAs (A = the strip's pooled queries from shared memory, B = pooled keys read from L2 as 16-byte
+// pieces), then takes two rows of the strip through the select.  Against separate score and list kernels
+// this saves a launch, a drain and a round trip of the scores through L2 on the latency chain behind the
+// pooling kernel.
+//   The channel order inside each group of 16 is permuted identically for both operands (lane t of a
+// quad holds channels 4t..4t+3 of the group and feeds them to two k-steps), which leaves every dot
+// product the same sum and lets each operand piece be one 16-byte load.
+// ------------------------------------------------------------------------------------------------
+constexpr int kStripRows = 16;
+
+template <int D>
+__host__ __device__ constexpr int strip_pitch(int NB) { return (NB + 31) / 32 * 32 + 4; }
+
+template <int D, int KPL>
+__global__ void __launch_bounds__(256) score_select_kernel(const float* __restrict__ qbar, const float* __restrict__ kbar,
+                                                           float* __restrict__ bs, const uint8_t* __restrict__ prot_blk,
+                                                           int H, int NB, float scale, int k_keep, int protect_rows,
+                                                           int protect_cols, int32_t* __restrict__ col_idx,
+                                                           int32_t* __restrict__ col_cnt) {
+  constexpr int PITCH = D + 4;
+  extern __shared__ __align__(16) float strip_smem[];
+  float* sq = strip_smem;                                   // [16][PITCH] pooled queries of the strip
+  const int SP = strip_pitch<D>(NB);
+  float* strip = sq + kStripRows * PITCH;                   // [16][SP] block scores of the strip
+  int* all_bins = reinterpret_cast<int*>(strip + kStripRows * SP);      // [8][256]
+  // Staged behind the pooling grid (programmatic dependent launch) and waits for it here; the pooling grid in
+  // turn retires only after the token select, so the block flags are final too.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int g = lane >> 2, t = lane & 3;
+  const int bh = blockIdx.y, i0 = blockIdx.x * kStripRows;
+  const float* qb = qbar + static_cast<int64_t>(bh) * NB * D;
+  const float* kb = kbar + static_cast<int64_t>(bh) * NB * D;
+  for (int e = tid; e < kStripRows * (D / 4); e += 256) {
+    const int r = e / (D / 4), c4 = e % (D / 4);
+    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (i0 + r < NB) v = __ldg(reinterpret_cast<const float4*>(qb + static_cast<int64_t>(i0 + r) * D) + c4);
+    *reinterpret_cast<float4*>(sq + r * PITCH + c4 * 4) = v;
+  }
+  __syncthreads();
+  for (int j0 = warp * 32; j0 < NB; j0 += 8 * 32) {
+    float acc[4][4];
+#pragma unroll
+    for (int ni = 0; ni < 4; ni++)
+#pragma unroll
+      for (int r = 0; r < 4; r++) acc[ni][r] = 0.f;
+    const float* krow[4];
+    bool kvalid[4];
+#pragma unroll
+    for (int ni = 0; ni < 4; ni++) {
+      const int col = j0 + ni * 8 + g;
+      kvalid[ni] = col < NB;
+      krow[ni] = kb + static_cast<int64_t>(kvalid[ni] ? col : 0) * D + 4 * t;
+    }
+#pragma unroll 4
+    for (int jg = 0; jg < D / 16; jg++) {
+      float4 kv[4];
+#pragma unroll
+      for (int ni = 0; ni < 4; ni++) {
+        kv[ni] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (kvalid[ni]) kv[ni] = __ldg(reinterpret_cast<const float4*>(krow[ni] + 16 * jg));
+      }
+      const float4 qa = *reinterpret_cast<const float4*>(sq + g * PITCH + 16 * jg + 4 * t);
+      const float4 qc = *reinterpret_cast<const float4*>(sq + (g + 8) * PITCH + 16 * jg + 4 * t);
+      // two k-steps: (x, y) and (z, w) of each piece
+      uint32_t ah[2][4], al[2][4];
+      split_tf32(qa.x, ah[0][0], al[0][0]);
+      split_tf32(qc.x, ah[0][1], al[0][1]);
+      split_tf32(qa.y, ah[0][2], al[0][2]);
+      split_tf32(qc.y, ah[0][3], al[0][3]);
+      split_tf32(qa.z, ah[1][0], al[1][0]);
+      split_tf32(qc.z, ah[1][1], al[1][1]);
+      split_tf32(qa.w, ah[1][2], al[1][2]);
+      split_tf32(qc.w, ah[1][3], al[1][3]);
+#pragma unroll
+      for (int ni = 0; ni < 4; ni++) {
+        uint32_t bhh[2][2], bl[2][2];
+        split_tf32(kv[ni].x, bhh[0][0], bl[0][0]);
+        split_tf32(kv[ni].y, bhh[0][1], bl[0][1]);
+        split_tf32(kv[ni].z, bhh[1][0], bl[1][0]);
+        split_tf32(kv[ni].w, bhh[1][1], bl[1][1]);
+#pragma unroll
+        for (int s2 = 0; s2 < 2; s2++) {
+          mma_tf32(acc[ni], al[s2], bhh[s2]);     // small terms first
+          mma_tf32(acc[ni], ah[s2], bl[s2]);
+          mma_tf32(acc[ni], ah[s2], bhh[s2]);
+        }
+      }
+    }
+#pragma unroll
+    for (int ni = 0; ni < 4; ni++) {
+      const int j = j0 + ni * 8 + 2 * t;
+      *reinterpret_cast<float2*>(strip + g * SP + j) = make_float2(acc[ni][0] * scale, acc[ni][1] * scale);
+      *reinterpret_cast<float2*>(strip + (g + 8) * SP + j) = make_float2(acc[ni][2] * scale, acc[ni][3] * scale);
+    }
+  }
+  __syncthreads();
+  const int b = bh / H;
+  const uint8_t* pb = prot_blk + static_cast<int64_t>(b) * NB;
+#pragma unroll 1
+  for (int rr = 0; rr < kStripRows / 8; rr++) {
+    const int r = warp * (kStripRows / 8) + rr;
+    const int qi = i0 + r;
+    if (qi >= NB) break;
+    const int64_t row = static_cast<int64_t>(bh) * NB + qi;
+    const float* src = strip + r * SP;
+    float* dst = bs + row * NB;
+    for (int i = lane; i < NB; i += 32) dst[i] = src[i];
+    select_row<KPL>(src, pb, protect_rows && pb[qi] != 0, NB, k_keep, protect_cols, all_bins + warp * 256, lane,
+                    col_idx + row * NB, col_cnt + row);
+  }
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -478,6 +516,43 @@ __global__ void __launch_bounds__(256) expand_blocks_kernel(const uint8_t* __res
   const int64_t b = idx / N;
   const int i = static_cast<int>(idx % N);
   prot_tok[idx] = prot_blk[b * NB + i / blk];
+}
+
+// Launches the fused score + list kernel with the key slots per lane that NB needs.
+template <int D>
+static cudaError_t launch_score_select(cudaLaunchConfig_t& cfg, int NB, const float* qbar, const float* kbar, float* bs,
+                                       const uint8_t* pblk, int H, float scale, int k_keep, int pr, int pc,
+                                       int32_t* col_idx, int32_t* col_cnt) {
+  const size_t smem = (static_cast<size_t>(kStripRows) * (D + 4) + static_cast<size_t>(kStripRows) * strip_pitch<D>(NB)) *
+                          sizeof(float) + 8 * 256 * sizeof(int);
+  cfg.blockDim = dim3(256, 1, 1);
+  cfg.dynamicSmemBytes = smem;
+  // always the same limit (the largest NB the call accepts), so concurrent callers never race on its value
+  constexpr int kMaxSmem = (kStripRows * (D + 4) + kStripRows * strip_pitch<D>(kMaxBlocksPerRow)) * 4 + 8 * 256 * 4;
+  cudaError_t e;
+  if (NB <= 256) {
+    e = cudaFuncSetAttribute(score_select_kernel<D, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
+    if (e != cudaSuccess) return e;
+    return cudaLaunchKernelEx(&cfg, score_select_kernel<D, 8>, qbar, kbar, bs, pblk, H, NB, scale, k_keep, pr, pc, col_idx,
+                              col_cnt);
+  }
+  if (NB <= 512) {
+    e = cudaFuncSetAttribute(score_select_kernel<D, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
+    if (e != cudaSuccess) return e;
+    return cudaLaunchKernelEx(&cfg, score_select_kernel<D, 16>, qbar, kbar, bs, pblk, H, NB, scale, k_keep, pr, pc,
+                              col_idx, col_cnt);
+  }
+  e = cudaFuncSetAttribute(score_select_kernel<D, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
+  if (e != cudaSuccess) return e;
+  return cudaLaunchKernelEx(&cfg, score_select_kernel<D, 64>, qbar, kbar, bs, pblk, H, NB, scale, k_keep, pr, pc, col_idx,
+                            col_cnt);
+}
+
+// The staged token select may use up to kSelectSmemKeys keys of dynamic shared memory.  The limit is always set
+// to that same maximum, so host threads that call with different N never race on the attribute's value.
+static bool allow_select_smem() {
+  return cudaFuncSetAttribute(token_select_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              static_cast<int>(kSelectSmemKeys * sizeof(uint32_t))) == cudaSuccess;
 }
 
 struct MaskWorkspace {
@@ -540,33 +615,30 @@ extern "C" int avsa_build_block_mask(int B, int H, int N, int d, int blk, avsa_b
     float* bsum = reinterpret_cast<float*>(base + w.bsum);
     if (n_protect > 0) block_sum_kernel<<<dim3((NB + 7) / 8, B), 256, 0, st>>>(scores, N, blk, NB, bsum);
     const size_t key_bytes = static_cast<size_t>(NB) * sizeof(uint32_t);
-    if (cudaFuncSetAttribute(token_select_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             static_cast<int>(key_bytes)) != cudaSuccess)
-      return AVSA_ERR_CUDA;
+    if (!allow_select_smem()) return AVSA_ERR_CUDA;
     token_select_kernel<true><<<B, 1024, key_bytes, st>>>(bsum, NB, n_protect, 32, (NB + 31) / 32, 1, pblk,
                                                          base + w.junk, static_cast<StatusRecord*>(ws));
   } else if (N <= kSelectSmemKeys) {
     const size_t key_bytes = static_cast<size_t>(N) * sizeof(uint32_t);
-    if (cudaFuncSetAttribute(token_select_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             static_cast<int>(key_bytes)) != cudaSuccess)
-      return AVSA_ERR_CUDA;
+    if (!allow_select_smem()) return AVSA_ERR_CUDA;
     token_select_kernel<true><<<B, 1024, key_bytes, st>>>(scores, N, n_protect, blk, NB, min_tokens, ptok, pblk,
                                                          static_cast<StatusRecord*>(ws));
   } else {
     token_select_kernel<false><<<B, 1024, 0, st>>>(scores, N, n_protect, blk, NB, min_tokens, ptok, pblk,
                                                    static_cast<StatusRecord*>(ws));
   }
+  const int total_rows = B * H * NB;
+  const int pr = (flags & AVSA_PROTECT_ROWS) ? 1 : 0, pc = (flags & AVSA_PROTECT_COLS) ? 1 : 0;
+  const uint8_t* pbc = pblk;
   if (!given) {
     const __nv_bfloat16* qp = static_cast<const __nv_bfloat16*>(q.ptr);
     const __nv_bfloat16* kp = static_cast<const __nv_bfloat16*>(k.ptr);
-    dim3 pg(NB, B * H, 2);
-    dim3 sg((NB + 63) / 64, (NB + 63) / 64, B * H);
     // the pooling kernel does not read anything the token select writes: allow it to start early
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = pg;
+    cfg.gridDim = dim3(NB, B * H, 2);
     cfg.blockDim = dim3(256, 1, 1);
     cfg.dynamicSmemBytes = 0;
     cfg.stream = st;
@@ -574,56 +646,32 @@ extern "C" int avsa_build_block_mask(int B, int H, int N, int d, int blk, avsa_b
     cfg.numAttrs = 1;
     const int64_t qsb = q.stride_b, qsh = q.stride_h, qsn = q.stride_n, ksb = k.stride_b, ksh = k.stride_h,
                   ksn = k.stride_n;
-    const size_t score_smem = static_cast<size_t>(2) * 64 * (d + 4) * sizeof(float);
     cudaError_t e;
-    if (d == 128) {
+    if (d == 128)
       e = cudaLaunchKernelEx(&cfg, pool_kernel<128>, qp, qsb, qsh, qsn, kp, ksb, ksh, ksn, qbar, kbar, H, N, blk);
-      if (e != cudaSuccess) return AVSA_ERR_CUDA;
-      if (cudaFuncSetAttribute(block_score_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                               static_cast<int>(score_smem)) != cudaSuccess)
-        return AVSA_ERR_CUDA;
-      cfg.gridDim = sg;
-      cfg.blockDim = dim3(128, 1, 1);
-      cfg.dynamicSmemBytes = score_smem;
-      const float* qbc = qbar;
-      const float* kbc = kbar;
-      e = cudaLaunchKernelEx(&cfg, block_score_kernel<128>, qbc, kbc, block_scores, NB, scale);
-      if (e != cudaSuccess) return AVSA_ERR_CUDA;
-    } else {
-      e = cudaLaunchKernelEx(&cfg, pool_kernel<64>, qp, qsb, qsh, qsn, kp, ksb, ksh, ksn, qbar, kbar, H, N, blk);
-      if (e != cudaSuccess) return AVSA_ERR_CUDA;
-      cfg.gridDim = sg;
-      cfg.blockDim = dim3(128, 1, 1);
-      cfg.dynamicSmemBytes = score_smem;
-      const float* qbc = qbar;
-      const float* kbc = kbar;
-      e = cudaLaunchKernelEx(&cfg, block_score_kernel<64>, qbc, kbc, block_scores, NB, scale);
-      if (e != cudaSuccess) return AVSA_ERR_CUDA;
-    }
-  }
-  const int total_rows = B * H * NB;
-  const int pr = (flags & AVSA_PROTECT_ROWS) ? 1 : 0, pc = (flags & AVSA_PROTECT_COLS) ? 1 : 0;
-  const unsigned rgrid = static_cast<unsigned>((total_rows + 3) / 4);
-  {
-    cudaLaunchAttribute rattr[1];
-    rattr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    rattr[0].val.programmaticStreamSerializationAllowed = given ? 0 : 1;   // only behind the block-score kernel
-    cudaLaunchConfig_t rcfg = {};
-    rcfg.gridDim = dim3(rgrid, 1, 1);
-    rcfg.blockDim = dim3(128, 1, 1);
-    rcfg.dynamicSmemBytes = 0;
-    rcfg.stream = st;
-    rcfg.attrs = rattr;
-    rcfg.numAttrs = 1;
-    const float* bsc = block_scores;
-    const uint8_t* pbc = pblk;
-    cudaError_t e;
-    if (NB <= 256)
-      e = cudaLaunchKernelEx(&rcfg, row_select_kernel<8>, bsc, pbc, H, NB, k_keep, pr, pc, total_rows, col_idx, col_cnt);
-    else if (NB <= 512)
-      e = cudaLaunchKernelEx(&rcfg, row_select_kernel<16>, bsc, pbc, H, NB, k_keep, pr, pc, total_rows, col_idx, col_cnt);
     else
-      e = cudaLaunchKernelEx(&rcfg, row_select_kernel<64>, bsc, pbc, H, NB, k_keep, pr, pc, total_rows, col_idx, col_cnt);
+      e = cudaLaunchKernelEx(&cfg, pool_kernel<64>, qp, qsb, qsh, qsn, kp, ksb, ksh, ksn, qbar, kbar, H, N, blk);
+    if (e != cudaSuccess) return AVSA_ERR_CUDA;
+    // block scores and lists of 16 query blocks per CTA, staged behind the pooling grid
+    cfg.gridDim = dim3((NB + kStripRows - 1) / kStripRows, B * H, 1);
+    const float* qbc = qbar;
+    const float* kbc = kbar;
+    if (d == 128)
+      e = launch_score_select<128>(cfg, NB, qbc, kbc, block_scores, pbc, H, scale, k_keep, pr, pc, col_idx, col_cnt);
+    else
+      e = launch_score_select<64>(cfg, NB, qbc, kbc, block_scores, pbc, H, scale, k_keep, pr, pc, col_idx, col_cnt);
+    if (e != cudaSuccess) return AVSA_ERR_CUDA;
+  } else {
+    const unsigned rgrid = static_cast<unsigned>((total_rows + 3) / 4);
+    const float* bsc = block_scores;
+    cudaError_t e = cudaSuccess;
+    if (NB <= 256)
+      row_select_kernel<8><<<rgrid, 128, 0, st>>>(bsc, pbc, H, NB, k_keep, pr, pc, total_rows, col_idx, col_cnt);
+    else if (NB <= 512)
+      row_select_kernel<16><<<rgrid, 128, 0, st>>>(bsc, pbc, H, NB, k_keep, pr, pc, total_rows, col_idx, col_cnt);
+    else
+      row_select_kernel<64><<<rgrid, 128, 0, st>>>(bsc, pbc, H, NB, k_keep, pr, pc, total_rows, col_idx, col_cnt);
+    e = cudaGetLastError();
     if (e != cudaSuccess) return AVSA_ERR_CUDA;
   }
   if (by_block_sum) {

@@ -120,14 +120,6 @@ static int launch_sparse_attn(int B, int H, int N, const avsa_bf16_4d& q, const 
 
 using namespace avsa;
 
-#ifdef AVSA_TRACE
-// Debug builds only: device buffer that receives the pipeline time stamps of CTA (0,0,0).
-static long long* g_trace_buffer = nullptr;
-extern "C" __attribute__((visibility("default"))) void avsa_debug_set_trace(long long* device_buffer) {
-  g_trace_buffer = device_buffer;
-}
-#endif
-
 extern "C" int avsa_selftest_bounded_wait(void* ws, size_t ws_bytes, long long limit_cycles, void* stream) {
   if (ws == nullptr || ws_bytes < kStatusBytes) return AVSA_ERR_WORKSPACE;
   if (limit_cycles < 0 || limit_cycles > 2000000000ll) return AVSA_ERR_INVALID_ARG;     // about a second at most
@@ -166,9 +158,6 @@ extern "C" int avsa_sparse_self_attn(int B, int H, int N, int d, int blk, avsa_b
   prm.NQT = prm.NKB = (N + blk - 1) / blk;
   const float scale = softmax_scale != 0.f ? softmax_scale : 1.0f / sqrtf(static_cast<float>(d));
   prm.scale_log2 = scale * 1.4426950408889634f;
-#ifdef AVSA_TRACE
-  prm.trace = g_trace_buffer;
-#endif
   int* redo = reinterpret_cast<int*>(static_cast<uint8_t*>(ws) + kStatusBytes);
   const long long n_items = static_cast<long long>(B) * H * prm.NQT;
   if (n_items > 0x3fffffff) return AVSA_ERR_UNSUPPORTED;

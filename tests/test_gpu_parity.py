@@ -3,7 +3,7 @@
 Bars: integer outputs (flags, lists, counts) bit-exact given the same fp32 score tensors.
 bf16 attention outputs O: relative-L2 5e-3 and max-abs 1e-2, the latter scaled by |value| above 1 (the bf16
 grid itself is coarser than 1e-2 there).  fp32 log-sum-exps: max-abs 1e-3, unscaled.  fp32 response scores
-(Eq. 2): every element within 5e-3 of its own value (plus 1e-6 of the largest score), so that a few wrong
+(Eq. 2): every element within 1e-3 of its own value (plus 1e-6 of the largest score), so that a few wrong
 columns cannot hide in a norm.
 """
 import numpy as np
