@@ -37,7 +37,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # summarised under profiles/ (None until a capture exists for that workload)
 NCU_TRAFFIC_BYTES = {"mid": 482.3e6,      # captured (profiles/attn_persist_kernel_mid.md)
                      "ovi": 861.1e6}      # captured on the full launch with the two DRAM counters only (same file)
-KERNELS_PER_STEP = 13   # cross: clear, pass 1, its redo pass, merge, pass 2, head sum; mask: select, pool, scores, rows; attn: prep, persistent, redo
+KERNELS_PER_STEP = 12   # cross: clear, pass 1, its redo pass, merge, pass 2, head sum; mask: select, pool, scores + lists; attn: prep, persistent, redo
 
 
 def load_peaks():
@@ -47,6 +47,36 @@ def load_peaks():
             p = json.load(f)
         return p, "measured"
     return dict(FALLBACK_PEAKS), "fallback"
+
+
+def static_config(w):
+    """What defines the workload (the same dict in both arms); data-dependent figures go to ``mask_stats``."""
+    nb = w.n_blocks
+    return {"workload": w.name, "B": w.B, "H": w.H, "d": w.d, "n_video": w.n_video, "n_audio": w.n_audio, "blk": w.blk,
+            "keep_pct": w.keep_pct, "protect_pct": w.protect_pct,
+            "k_keep": max(1, (w.keep_pct * nb + 99) // 100), "n_protect": (w.protect_pct * w.n_video + 99) // 100,
+            "n_blocks": nb,
+            "l2": "inputs (Q,K,V of both attentions) are larger than the 126 MB L2; no flush",
+            "multi_gpu": "independent replica per GPU, no data-path collective"}
+
+
+def cross_roofline(w, t_fwd_ms, t_rev_ms, peak_tflops, hbm_gbs):
+    """The cross-attention call sits at the ridge (N_a FLOP per byte of K and V), so both fractions are given: the
+    time the tensor cores need for its 6 H N_a N_v d FLOPs (4 in pass 1, 2 in pass 2) at the measured bf16 peak, and
+    the time to stream K and V once at the measured copy bandwidth, each over the measured time; the larger one
+    binds.  The reverse direction (video queries, audio keys) streams Q once and has the same FLOPs."""
+    flops = 6.0 * w.B * w.H * w.n_audio * float(w.n_video) * w.d
+    out = {}
+    for tag, t_ms, nbytes in (("forward", t_fwd_ms, 2.0 * w.B * w.H * w.n_video * w.d * 2),
+                              ("reverse", t_rev_ms, 2.0 * w.B * w.H * w.n_video * w.d * 2)):
+        t_tc = flops / (peak_tflops * 1e12) * 1e3
+        t_hbm = nbytes / (hbm_gbs * 1e9) * 1e3
+        out[tag] = {"ms": t_ms, "tflops": flops / (t_ms * 1e-3) / 1e12, "gbs": nbytes / (t_ms * 1e-3) / 1e9,
+                    "frac_of_bf16_peak": t_tc / t_ms, "frac_of_hbm_peak": t_hbm / t_ms,
+                    "binding": "tensor" if t_tc >= t_hbm else "hbm", "frac_of_binding_roofline": max(t_tc, t_hbm) / t_ms}
+    out["note"] = ("forward: inside the step loop; reverse: 10 launches in a row outside it; reverse bytes = Q (video) "
+                   "read by both passes from HBM/L2 once plus O written")
+    return out
 
 
 def dense_flops(w):
@@ -219,18 +249,21 @@ def run_reference(args, w):
     cores = len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else os.cpu_count()
     for _ in range(min(args.warmup, 1)):
         oracle_sample(w, q_blocks=2)
-    times, desc = [], ""
+    times, measured, desc = [], [], ""
     for _ in range(max(1, args.steps)):
-        t, desc, _ = oracle_sample(w, q_blocks=32)
+        t, desc, t_meas = oracle_sample(w, q_blocks=32)
         times.append(t)
+        measured.append(t_meas)
     t_layer = float(np.median(times))
     value = dense_flops(w) / t_layer / 1e12
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": t_layer * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": w.name, "keep_pct": w.keep_pct, "protect_pct": w.protect_pct},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc},
+        "config": static_config(w),
+        "extrapolated": True, "measured_s": float(np.median(measured)),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": desc,
+                         "extrapolated": True, "measured_s": float(np.median(measured))},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -344,6 +377,12 @@ def run_ours(args, w):
     except Exception:
         t_dense_lib = None
     t_token_exact = time_fn(token_exact_attn, reps)
+    # ---- reverse direction of the bidirectional pair (video queries, audio keys): audio-token saliency
+    gamma_r = 1.0 / (w.H * w.n_video)
+    o_r, lse_r, s_r, ws_r = av.avsa_cross_attn_scores(kc, qa, qa, score_gamma=gamma_r)
+    t_cross_rev = time_fn(lambda: av.avsa_cross_attn_scores(kc, qa, qa, scores=s_r, score_gamma=gamma_r, o=o_r, lse=lse_r,
+                                                            ws=ws_r), 10)
+    del o_r, lse_r, s_r, ws_r
     # ---- cache-reuse indicators (Eq. 12-15) on feature maps of the layer's size ([B, N, H*d] views of Q/K buffers)
     C = w.H * w.d
     yv, yhv = q.view(w.B, w.n_video, C), k.view(w.B, w.n_video, C)
@@ -418,6 +457,15 @@ def run_ours(args, w):
     e2e_ms = time_e2e(e2e_pipelined, e2e_steps)
     del sets
 
+    # ---- the other configurations (one GPU, default workload only), outside the headline timed region
+    extras = None
+    if rank == 0 and world == 1 and w.name == "ovi" and not args.no_extras:
+        del host_in, host_out, q, k, v, qa, kc, vc, o, o_tok, yv, yhv, ya, yha
+        torch.cuda.empty_cache()
+        peaks_x, _ = load_peaks()
+        extras = run_extras(av, dev, float(peaks_x.get("bf16_tflops", FALLBACK_PEAKS["bf16_tflops"])),
+                            float(peaks_x.get("hbm_gbs", FALLBACK_PEAKS["hbm_gbs"])))
+
     # ---- max over ranks
     total_ms, e2e_ms, e2e_serial_ms = dt.max_over_ranks(dist, [total_ms, e2e_ms, e2e_serial_ms], dev)
     ms_per_step = total_ms / args.steps
@@ -443,16 +491,13 @@ def run_ours(args, w):
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": w.name, "B": w.B, "H": w.H, "d": w.d, "n_video": w.n_video, "n_audio": w.n_audio,
-                       "blk": w.blk, "keep_pct": w.keep_pct, "protect_pct": w.protect_pct, "k_keep": k_keep,
-                       "n_protect": n_protect, "protected_blocks": prot_blocks, "n_blocks": NB,
-                       "executed_pair_fraction": pairs / float(w.B * w.H * NB * NB),
-                       # Eq. 16 beside it: kappa + rho on tokens, and kappa + p_b (1 - kappa) with p_b the
-                       # protected-BLOCK fraction (what block-level protection can reach at best)
-                       "eq16_kappa_plus_rho": (w.keep_pct + w.protect_pct) / 100.0,
-                       "eq16_kappa_plus_pb": k_keep / float(NB) + prot_blocks / float(w.B * NB) * (1.0 - k_keep / float(NB)),
-                       "l2": "inputs (Q,K,V of both attentions, 1.2 GB) are larger than the 126 MB L2; no flush",
-                       "multi_gpu": "independent replica per GPU, no data-path collective"},
+            "config": static_config(w),
+            "mask_stats": {"protected_blocks": prot_blocks, "n_blocks": NB,
+                           "executed_pair_fraction": pairs / float(w.B * w.H * NB * NB),
+                           # Eq. 16 beside it: kappa + rho on tokens, and kappa + p_b (1 - kappa) with p_b the
+                           # protected-BLOCK fraction (what block-level protection can reach at best)
+                           "eq16_kappa_plus_rho": (w.keep_pct + w.protect_pct) / 100.0,
+                           "eq16_kappa_plus_pb": k_keep / float(NB) + prot_blocks / float(w.B * NB) * (1.0 - k_keep / float(NB))},
             "ms": {"cross_attn_scores": t_cross, "build_block_mask": t_mask, "sparse_self_attn": t_attn,
                    "dense_keep_all_ours": t_dense_ours, "dense_library_sdpa": t_dense_lib,
                    "step_median": float(np.median(step_ms)), "step_min": float(np.min(step_ms)),
@@ -478,6 +523,7 @@ def run_ours(args, w):
                          "peak_source": f"{peak_kind} bf16_tflops (burst)", "frac_of_sustained": achieved / sustained,
                          "frac_of_nominal_2250": achieved / 2250.0,
                          "traffic": NCU_TRAFFIC_BYTES.get(w.name)},
+            "cross_attn": cross_roofline(w, t_cross, t_cross_rev, peak, hbm),
             "hbm_kernels": {"build_block_mask_gbs": mask_bytes / (t_mask * 1e-3) / 1e9,
                             "build_block_mask_frac": mask_bytes / (t_mask * 1e-3) / 1e9 / hbm,
                             "cross_attn_scores_gbs": cross_bytes / (t_cross * 1e-3) / 1e9,
@@ -492,6 +538,7 @@ def run_ours(args, w):
                             "is copy -> compute -> copy back with no overlap"},
             "gpu_launches": KERNELS_PER_STEP * args.steps,
             "clocks": clocks,
+            "extra": extras,
         }
         print(json.dumps(line))
     if dist is not None:
@@ -499,7 +546,7 @@ def run_ours(args, w):
         dist.destroy_process_group()
 
 
-def time_layer_step(av, w, seed, dev, n_iter=3, token_exact=False):
+def time_layer_step(av, w, seed, dev, n_iter=3, token_exact=False, n_dense=1):
     """Per-call CUDA-event times (ms, median of n_iter) of one layer-step on freshly generated tensors."""
     q, k, v = wl.make_self_qkv(w, seed, dev)
     qa, kc, vc = wl.make_cross_qkv(w, seed, dev)
@@ -532,23 +579,27 @@ def time_layer_step(av, w, seed, dev, n_iter=3, token_exact=False):
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         torch.nn.functional.scaled_dot_product_attention(q, k, v)
         a.record()
-        torch.nn.functional.scaled_dot_product_attention(q, k, v)
+        for _ in range(n_dense):
+            torch.nn.functional.scaled_dot_product_attention(q, k, v)
         b.record(); torch.cuda.synchronize()
-        t_dense = a.elapsed_time(b)
+        t_dense = a.elapsed_time(b) / n_dense
     except Exception:
         pass
     NB = w.n_blocks
     pairs = int(m["col_cnt"].sum().item())
     executed = (pairs * w.blk * w.blk + (w.B * w.H * n_protect * float(w.n_video) if token_exact else 0.0)) / (
         w.B * w.H * float(w.n_video) ** 2)
+    fl_exec = executed * dense_flops(w)
     return {"cross_ms": float(t[0]), "mask_ms": float(t[1]), "sparse_ms": float(t[2]), "protected_rows_ms": float(t[3]),
-            "attn_ms": float(t[2] + t[3]), "dense_library_ms": t_dense, "executed_fraction": executed,
+            "attn_ms": float(t[2] + t[3]), "step_ms": float(t.sum()), "dense_library_ms": t_dense,
+            "executed_fraction": executed, "executed_tflops": fl_exec / (float(t[2] + t[3]) * 1e-3) / 1e12,
             "protected_blocks": int(m["prot_blk"].sum().item()), "n_blocks": NB}
 
 
 def run_single_call(args, w):
     """Times ONE call of the path alone on the chosen workload (its inputs come from the other calls, run once
-    before): ``--call cross | cross_rev | mask | attn | rows``.  This is also the command the per-call ncu
+    before): ``--call cross | cross_rev | mask | attn | rows``, the dense special case of the attention call
+    (``dense``: keep-all lists) or the library's dense attention on the same tensors (``dense_lib``).  This is also the command the per-call ncu
     captures under profiles/ run, since it launches little besides the kernels of that call."""
     from paper_2608_15522_b200 import binding as av
     dev = torch.device("cuda", 0)
@@ -572,6 +623,13 @@ def run_single_call(args, w):
         fn = lambda: av.avsa_build_block_mask(q, k, s, n_protect, k_keep, w.blk, flags=flags, out=m, ws=m["ws"])
     elif args.call == "attn":
         fn = lambda: av.avsa_sparse_self_attn(q, k, v, m["col_idx"], m["col_cnt"], w.blk, o=o, ws=ws3)
+    elif args.call == "dense":
+        NB = w.n_blocks
+        idx_all = torch.arange(NB, dtype=torch.int32, device=dev).expand(w.B, w.H, NB, NB).contiguous()
+        cnt_all = torch.full((w.B, w.H, NB), NB, dtype=torch.int32, device=dev)
+        fn = lambda: av.avsa_sparse_self_attn(q, k, v, idx_all, cnt_all, w.blk, o=o, ws=ws3)
+    elif args.call == "dense_lib":
+        fn = lambda: torch.nn.functional.scaled_dot_product_attention(q, k, v)
     else:
         ws4 = av.avsa_protected_rows_attn(q, k, v, m["prot_tok"], n_protect, w.blk, o)
         fn = lambda: av.avsa_protected_rows_attn(q, k, v, m["prot_tok"], n_protect, w.blk, o, ws=ws4)
@@ -589,6 +647,64 @@ def run_single_call(args, w):
         times.append(a.elapsed_time(b))
     print(json.dumps({"call": args.call, "workload": w.name, "steps": args.steps, "ms_median": float(np.median(times)),
                       "ms_min": float(np.min(times)), "l2": "256 MB written between timed launches"}))
+
+
+def run_extras(av, dev, peak_tflops, hbm_gbs):
+    """The other benchmark configurations, each over a few steps and with its own clock record: the LTX-class layer
+    (block mask and token-exact protection), three points of the mid-length sweep, and a shortened multi-step loop
+    on the Ovi-class shapes (fresh tensors and a rebuilt mask per layer-step)."""
+    out = {}
+
+    def sampled(fn):
+        smp = ClockSampler(dev.index or 0)
+        smp.start()
+        smp.begin()
+        r = fn()
+        torch.cuda.synchronize()
+        smp.end()
+        c = smp.stop()
+        r["clocks"] = {"sm_mhz": c.get("sm_mhz"), "sm_min_mhz": c.get("sm_min_mhz"), "reasons": c.get("reasons")}
+        return r
+
+    def layer(w, token_exact, n_iter=5):
+        r = time_layer_step(av, w, 0, dev, n_iter=n_iter, token_exact=token_exact, n_dense=n_iter)
+        r["attn_frac_of_bf16_peak"] = r["executed_tflops"] / peak_tflops
+        mask_bytes = 2.0 * w.B * w.H * w.n_video * w.d * 2 + 3.0 * w.B * w.H * w.n_blocks * w.n_blocks * 4
+        r["mask_frac_of_hbm_peak"] = mask_bytes / (r["mask_ms"] * 1e-3) / 1e9 / hbm_gbs
+        if r["dense_library_ms"]:
+            r["attn_speedup_vs_dense_library"] = r["dense_library_ms"] / r["attn_ms"]
+        r["protection"] = "tokens" if token_exact else "blocks"
+        return r
+
+    ltx = wl.WORKLOADS["ltx"]
+    out["ltx"] = {"config": static_config(ltx), "blocks": sampled(lambda: layer(ltx, False)),
+                  "tokens": sampled(lambda: layer(ltx, True))}
+    mid = wl.WORKLOADS["mid"]
+    out["mid_sweep"] = []
+    for keep, prot in ((10, 0), (25, 5), (50, 20)):
+        wm = mid.with_ratios(keep, prot)
+        row = {"keep_pct": keep, "protect_pct": prot, "blocks": sampled(lambda: layer(wm, False))}
+        if prot:
+            row["tokens"] = sampled(lambda: layer(wm, True))
+        out["mid_sweep"].append(row)
+    ovi = wl.WORKLOADS["ovi"]
+
+    def loop(token_exact, steps=2, layers=4):
+        tot = {"cross_ms": 0.0, "mask_ms": 0.0, "sparse_ms": 0.0, "protected_rows_ms": 0.0, "dense_library_ms": 0.0}
+        for st in range(steps):
+            for ly in range(layers):
+                r = time_layer_step(av, ovi, wl.loop_seed(st, ly), dev, n_iter=1, token_exact=token_exact)
+                for key in tot:
+                    tot[key] += r[key] or 0.0
+        ours = tot["cross_ms"] + tot["mask_ms"] + tot["sparse_ms"] + tot["protected_rows_ms"]
+        return {"steps": steps, "layers": layers, "ours_ms": ours, "dense_library_ms": tot["dense_library_ms"],
+                "speedup_vs_dense_library": tot["dense_library_ms"] / ours if ours else None,
+                "share": {k: v / ours for k, v in tot.items() if k != "dense_library_ms"},
+                "note": "the 8 x 30 loop of the benchmark plan cut to steps x layers layer-steps; "
+                        "`bench.py --loop` runs it in full"}
+
+    out["loop_ovi"] = {"blocks": sampled(lambda: loop(False)), "tokens": sampled(lambda: loop(True))}
+    return out
 
 
 def run_sweep(args, w):
@@ -697,9 +813,10 @@ def main():
     ap.add_argument("--workload", default="ovi", choices=wl.all_workload_names())
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extras", action="store_true", help="skip the other configurations (ltx, mid sweep, short loop)")
     ap.add_argument("--keep-pct", type=int, default=None)
     ap.add_argument("--protect-pct", type=int, default=None)
-    ap.add_argument("--call", default=None, choices=["cross", "cross_rev", "mask", "attn", "rows"],
+    ap.add_argument("--call", default=None, choices=["cross", "cross_rev", "mask", "attn", "rows", "dense", "dense_lib"],
                     help="time one call of the path alone (L2 flushed between launches)")
     ap.add_argument("--sweep", action="store_true", help="keep x protect grid on the chosen workload (one JSON line)")
     ap.add_argument("--loop", action="store_true", help="multi-step denoising loop on the chosen workload")

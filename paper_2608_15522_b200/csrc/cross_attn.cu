@@ -83,8 +83,9 @@ colsum_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ C
     prefetch_tmap(&tmq);
     prefetch_tmap(&tmk);
   }
+  // negated log2-domain LSEs (one packed FMA then gives s*c - lse2); queries beyond Nq get -inf: exp2 = 0
   for (int j = tid; j < NCH * W; j += kColThreads)
-    lse2[j] = (j < p.Nq) ? p.lse[(static_cast<int64_t>(b) * p.H + h) * p.Nq + j] * 1.4426950408889634f : INFINITY;
+    lse2[j] = (j < p.Nq) ? -p.lse[(static_cast<int64_t>(b) * p.H + h) * p.Nq + j] * 1.4426950408889634f : -INFINITY;
   if (warp == 2) {
     tmem_alloc(smem_u32(const_cast<uint32_t*>(misc)), 512);
     tmem_relinquish();
@@ -122,29 +123,40 @@ colsum_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ C
       }
     }
   } else if (warp == 1) {
-    if (lane == 0) {
-      const uint32_t idesc = make_idesc_bf16(128, W, 0, 0);
-      bool ok = wait_or_abort(Q_FULL, 0, kColQFull, 0);
-      for (int t = 0; t < ntile && ok; t++) {
-        const int s = t % kColStages, f = t / kColStages;
-        ok = wait_or_abort(K_FULL + s, f & 1, kColKFull, t);
+    // The whole warp runs the loop (uniform control flow), one elected lane issues; descriptor words are
+    // prepared ahead so that the issuing lane does little besides issuing.
+    const bool leader = elect_one_sync();
+    const uint32_t idesc = make_idesc_bf16(128, W, 0, 0);
+    constexpr uint32_t desc_hi = (1024u >> 4) | (1u << 14) | (2u << 29);
+    auto desc64 = [](uint32_t lo) { return (static_cast<uint64_t>(desc_hi) << 32) | lo; };
+    const uint32_t k_lo0 = ((smem_u32(smem + L::kK) & 0x3FFFFu) >> 4) | (1u << 16);
+    const uint32_t q_lo0 = ((smem_u32(smem + L::kQ) & 0x3FFFFu) >> 4) | (1u << 16);
+    auto wait_all = [&](int bar, uint32_t parity, int where, int aux) -> bool {
+      return __all_sync(0xffffffffu, wait_or_abort(bar, parity, where, aux));
+    };
+    bool ok = wait_all(Q_FULL, 0, kColQFull, 0);
+    for (int t = 0; t < ntile && ok; t++) {
+      const int s = t % kColStages, f = t / kColStages;
+      ok = wait_all(K_FULL + s, f & 1, kColKFull, t);
+      if (!ok) break;
+      const uint32_t k_lo = k_lo0 + s * (L::kKTile >> 4);
+      for (int ch = 0; ch < NCH && ok; ch++) {
+        const int u = t * NCH + ch, g = u & 1, i = u >> 1;
+        if (i > 0) ok = wait_all(S_EMPTY + g, (i - 1) & 1, kColSEmpty, u);
         if (!ok) break;
-        const uint32_t k_addr = smem_u32(smem + L::kK) + s * L::kKTile;
-        for (int ch = 0; ch < NCH && ok; ch++) {
-          const int u = t * NCH + ch, g = u & 1, i = u >> 1;
-          if (i > 0) ok = wait_or_abort(S_EMPTY + g, (i - 1) & 1, kColSEmpty, u);
-          if (!ok) break;
-          tc_fence_after();
-          const uint32_t q_addr = smem_u32(smem + L::kQ) + ch * q_chunk_bytes;
+        tc_fence_after();
+        const uint32_t q_lo = q_lo0 + ch * (q_chunk_bytes >> 4);
+        if (leader) {
 #pragma unroll
           for (int ks = 0; ks < D / 16; ks++) {
-            const uint64_t ad = make_sdesc(k_addr + (ks >> 2) * KPANEL_BYTES + (ks & 3) * 32, 16, 1024);
-            const uint64_t bd = make_sdesc(q_addr + (ks >> 2) * q_panel_bytes + (ks & 3) * 32, 16, 1024);
-            umma_ss(tmem + g * 256, ad, bd, idesc, ks > 0 ? 1u : 0u);
+            const uint32_t koff = ((ks >> 2) * KPANEL_BYTES + (ks & 3) * 32) >> 4;
+            const uint32_t qoff = ((ks >> 2) * q_panel_bytes + (ks & 3) * 32) >> 4;
+            umma_ss(tmem + g * 256, desc64(k_lo + koff), desc64(q_lo + qoff), idesc, ks > 0 ? 1u : 0u);
           }
           umma_commit(BAR(S_FULL + g));
+          if (ch == NCH - 1) umma_commit(BAR(K_EMPTY + s));
         }
-        if (ok) umma_commit(BAR(K_EMPTY + s));
+        __syncwarp();
       }
     }
   } else if (warp >= 4) {
@@ -158,35 +170,49 @@ colsum_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ C
       if (!ok) break;
       tc_fence_after();
       const float* l2 = lse2 + ch * W;
-      float sum0 = 0.f, sum1 = 0.f;
       const uint32_t base = tmem + g * 256 + lane_off;
-      int c = 0;
-      for (; c + 32 <= W; c += 32) {
-        uint32_t s[32];
-        tmem_ld32(base + c, s);
-        tmem_wait_ld();
+      const uint64_t c2 = pack_f32x2(p.scale_log2, p.scale_log2);
+      uint64_t acc[4] = {0ull, 0ull, 0ull, 0ull};
+      // sum over 32 (or 16) queries of exp2(s*c - lse2), two values per packed FMA / add
+      auto reduce32 = [&](const uint32_t (&sv)[32], const float* nl) {
 #pragma unroll
         for (int j = 0; j < 32; j += 4) {
-          const float4 lv = *reinterpret_cast<const float4*>(l2 + c + j);
-          sum0 += fast_exp2(fmaf(__uint_as_float(s[j]), p.scale_log2, -lv.x));
-          sum1 += fast_exp2(fmaf(__uint_as_float(s[j + 1]), p.scale_log2, -lv.y));
-          sum0 += fast_exp2(fmaf(__uint_as_float(s[j + 2]), p.scale_log2, -lv.z));
-          sum1 += fast_exp2(fmaf(__uint_as_float(s[j + 3]), p.scale_log2, -lv.w));
+          const ulonglong2 nv = *reinterpret_cast<const ulonglong2*>(nl + j);      // four negated LSEs
+          float x0, x1, x2, x3;
+          unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(sv[j]), __uint_as_float(sv[j + 1])), c2, nv.x), x0, x1);
+          unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(sv[j + 2]), __uint_as_float(sv[j + 3])), c2, nv.y), x2, x3);
+          acc[(j >> 2) & 3] = add_f32x2(acc[(j >> 2) & 3], pack_f32x2(fast_exp2(x0), fast_exp2(x1)));
+          acc[((j >> 2) + 2) & 3] = add_f32x2(acc[((j >> 2) + 2) & 3], pack_f32x2(fast_exp2(x2), fast_exp2(x3)));
         }
-      }
-      if (c < W) {   // W is a multiple of 16
-        uint32_t s[16];
-        tmem_ld16(base + c, s);
+      };
+      const int n32 = W / 32;           // whole 32-column pieces; W is a multiple of 16, so 16 columns may remain
+      uint32_t sa[32], sb[32];
+      if (n32 > 0) tmem_ld32(base, sa);
+      for (int c = 0; c < n32; c += 2) {
         tmem_wait_ld();
-#pragma unroll
-        for (int j = 0; j < 16; j += 4) {
-          const float4 lv = *reinterpret_cast<const float4*>(l2 + c + j);
-          sum0 += fast_exp2(fmaf(__uint_as_float(s[j]), p.scale_log2, -lv.x));
-          sum1 += fast_exp2(fmaf(__uint_as_float(s[j + 1]), p.scale_log2, -lv.y));
-          sum0 += fast_exp2(fmaf(__uint_as_float(s[j + 2]), p.scale_log2, -lv.z));
-          sum1 += fast_exp2(fmaf(__uint_as_float(s[j + 3]), p.scale_log2, -lv.w));
+        if (c + 1 < n32) tmem_ld32(base + (c + 1) * 32, sb);      // in flight under the exponentials of piece c
+        reduce32(sa, l2 + c * 32);
+        if (c + 1 < n32) {
+          tmem_wait_ld();
+          if (c + 2 < n32) tmem_ld32(base + (c + 2) * 32, sa);
+          reduce32(sb, l2 + (c + 1) * 32);
         }
       }
+      if (n32 * 32 < W) {
+        uint32_t st[16];
+        tmem_ld16(base + n32 * 32, st);
+        tmem_wait_ld();
+        const float* nl = l2 + n32 * 32;
+#pragma unroll
+        for (int j = 0; j < 16; j += 2) {
+          float x0, x1;
+          unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(st[j]), __uint_as_float(st[j + 1])), c2,
+                                 *reinterpret_cast<const uint64_t*>(nl + j)), x0, x1);
+          acc[(j >> 1) & 3] = add_f32x2(acc[(j >> 1) & 3], pack_f32x2(fast_exp2(x0), fast_exp2(x1)));
+        }
+      }
+      float sum0, sum1;
+      unpack_f32x2(add_f32x2(add_f32x2(acc[0], acc[1]), add_f32x2(acc[2], acc[3])), sum0, sum1);
       tc_fence_before();
       mbar_arrive(BAR(S_EMPTY + g));
       const int key = (kt0 + t) * 128 + row;
@@ -212,7 +238,7 @@ constexpr int kRevStages = 3;
 constexpr int kRevLseSlots = 5;      // LSE slices outlive their query stage by up to two units of exponentials
 
 struct ColsumRevParams {
-  const float* lse2;       // [B,H,NQC*128] log2-domain LSE, +inf beyond Nq
+  const float* lse2;       // [B,H,NQC*128] negated log2-domain LSE, -inf beyond Nq
   float* partial;          // [n_range*2][B,H,Nk]
   StatusRecord* status;
   int H, Nk, NKT, NQC;     // key tiles (<= 4) and query chunks of 128
@@ -351,23 +377,37 @@ colsum_rev_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant
       ok = wait_or_abort(S_FULL + g, i & 1, kRevSFull, u);
       if (!ok) break;
       tc_fence_after();
-      const float* l2 = lse_slots + (c % kRevLseSlots) * 128;
-      float sum0 = 0.f, sum1 = 0.f;
+      const float* l2 = lse_slots + (c % kRevLseSlots) * 128;       // negated log2-domain LSEs of the chunk's queries
       const uint32_t base = tmem + g * 128 + lane_off;
-#pragma unroll
-      for (int cc = 0; cc < 128; cc += 32) {
-        uint32_t s[32];
-        tmem_ld32(base + cc, s);
-        tmem_wait_ld();
+      const uint64_t c2 = pack_f32x2(p.scale_log2, p.scale_log2);
+      uint64_t acc2[4] = {0ull, 0ull, 0ull, 0ull};
+      auto reduce32 = [&](const uint32_t (&sv)[32], const float* nl) {
 #pragma unroll
         for (int j = 0; j < 32; j += 4) {
-          const float4 lv = *reinterpret_cast<const float4*>(l2 + cc + j);
-          sum0 += fast_exp2(fmaf(__uint_as_float(s[j]), p.scale_log2, -lv.x));
-          sum1 += fast_exp2(fmaf(__uint_as_float(s[j + 1]), p.scale_log2, -lv.y));
-          sum0 += fast_exp2(fmaf(__uint_as_float(s[j + 2]), p.scale_log2, -lv.z));
-          sum1 += fast_exp2(fmaf(__uint_as_float(s[j + 3]), p.scale_log2, -lv.w));
+          const ulonglong2 nv = *reinterpret_cast<const ulonglong2*>(nl + j);
+          float x0, x1, x2, x3;
+          unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(sv[j]), __uint_as_float(sv[j + 1])), c2, nv.x), x0, x1);
+          unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(sv[j + 2]), __uint_as_float(sv[j + 3])), c2, nv.y), x2, x3);
+          acc2[(j >> 2) & 3] = add_f32x2(acc2[(j >> 2) & 3], pack_f32x2(fast_exp2(x0), fast_exp2(x1)));
+          acc2[((j >> 2) + 2) & 3] = add_f32x2(acc2[((j >> 2) + 2) & 3], pack_f32x2(fast_exp2(x2), fast_exp2(x3)));
         }
-      }
+      };
+      // the next 32 columns are in flight under the exponentials of the current ones
+      uint32_t sa[32], sb[32];
+      tmem_ld32(base, sa);
+      tmem_wait_ld();
+      tmem_ld32(base + 32, sb);
+      reduce32(sa, l2);
+      tmem_wait_ld();
+      tmem_ld32(base + 64, sa);
+      reduce32(sb, l2 + 32);
+      tmem_wait_ld();
+      tmem_ld32(base + 96, sb);
+      reduce32(sa, l2 + 64);
+      tmem_wait_ld();
+      reduce32(sb, l2 + 96);
+      float sum0, sum1;
+      unpack_f32x2(add_f32x2(add_f32x2(acc2[0], acc2[1]), add_f32x2(acc2[2], acc2[3])), sum0, sum1);
       tc_fence_before();
       mbar_arrive(BAR(S_EMPTY + g));
       const float tot = sum0 + sum1;
@@ -386,13 +426,13 @@ colsum_rev_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant
   if (warp == 2) tmem_dealloc(tmem, 256);
 }
 
-// lse2[bh][i] = lse[bh][i] * log2(e) for i < Nq, +inf up to the padded length (multiple of 128)
+// lse2[bh][i] = -lse[bh][i] * log2(e) for i < Nq (negated: one FMA gives s*c - lse2), -inf up to the padded length
 __global__ void __launch_bounds__(256) lse_to_log2_kernel(const float* __restrict__ lse, int Nq, int Nq_pad, int BH,
                                                           float* __restrict__ lse2) {
   const int64_t idx = static_cast<int64_t>(blockIdx.x) * 256 + threadIdx.x;
   if (idx >= static_cast<int64_t>(BH) * Nq_pad) return;
   const int bh = static_cast<int>(idx / Nq_pad), i = static_cast<int>(idx % Nq_pad);
-  lse2[idx] = i < Nq ? lse[static_cast<int64_t>(bh) * Nq + i] * 1.4426950408889634f : INFINITY;
+  lse2[idx] = i < Nq ? -lse[static_cast<int64_t>(bh) * Nq + i] * 1.4426950408889634f : -INFINITY;
 }
 
 // scores[b,i] = beta * scores[b,i] + gamma * sum_h sum_ch partial[ch][b,h,i], heads in ascending order

@@ -373,9 +373,9 @@ __global__ void __launch_bounds__(128) row_select_kernel(const float* __restrict
 // ------------------------------------------------------------------------------------------------
 // (ii)+(iv) fused: block scores Bs[bh, i, j] = qbar[bh,i,:] . kbar[bh,j,:] * scale for a strip of 16 query
 // blocks against every key block, kept in shared memory, then the lists of those 16 rows straight from
-// there.  One CTA of 8 warps per strip: each warp computes 32-column chunks of the strip with 3xTF32
-// m16n8k8 MMAs (A = the strip's pooled queries from shared memory, B = pooled keys read from L2 as 16-byte
-// pieces), then takes two rows of the strip through the select.  Against separate score and list kernels
+// there.  One CTA of 8 warps per strip: each warp computes 32-column chunks of the strip with 3xTF32 m16n8k8 MMAs
+// (A = the strip's pooled queries from shared memory, B = pooled keys read from L2 as 16-byte pieces), then takes
+// two rows of the strip through the select (about a thousand instructions per row).  Against separate score and list kernels
 // this saves a launch, a drain and a round trip of the scores through L2 on the latency chain behind the
 // pooling kernel.
 //   The channel order inside each group of 16 is permuted identically for both operands (lane t of a
@@ -387,18 +387,20 @@ constexpr int kStripRows = 16;
 template <int D>
 __host__ __device__ constexpr int strip_pitch(int NB) { return (NB + 31) / 32 * 32 + 4; }
 
-template <int D, int KPL>
-__global__ void __launch_bounds__(256) score_select_kernel(const float* __restrict__ qbar, const float* __restrict__ kbar,
-                                                           float* __restrict__ bs, const uint8_t* __restrict__ prot_blk,
-                                                           int H, int NB, float scale, int k_keep, int protect_rows,
-                                                           int protect_cols, int32_t* __restrict__ col_idx,
-                                                           int32_t* __restrict__ col_cnt) {
+template <int D, int KPL, int WARPS>
+__global__ void __launch_bounds__(WARPS * 32) score_select_kernel(const float* __restrict__ qbar, const float* __restrict__ kbar,
+                                                                  float* __restrict__ bs, const uint8_t* __restrict__ prot_blk,
+                                                                  int H, int NB, float scale, int k_keep, int protect_rows,
+                                                                  int protect_cols, int32_t* __restrict__ col_idx,
+                                                                  int32_t* __restrict__ col_cnt) {
   constexpr int PITCH = D + 4;
+  constexpr int NT = 32 / WARPS;              // 8-column MMA tiles per warp and pass: 4 with 8 warps, 2 with 16
+  constexpr int CHUNK = NT * 8;               // columns per warp and pass
   extern __shared__ __align__(16) float strip_smem[];
   float* sq = strip_smem;                                   // [16][PITCH] pooled queries of the strip
   const int SP = strip_pitch<D>(NB);
   float* strip = sq + kStripRows * PITCH;                   // [16][SP] block scores of the strip
-  int* all_bins = reinterpret_cast<int*>(strip + kStripRows * SP);      // [8][256]
+  int* all_bins = reinterpret_cast<int*>(strip + kStripRows * SP);      // [WARPS][256]
   // Staged behind the pooling grid (programmatic dependent launch) and waits for it here; the pooling grid in
   // turn retires only after the token select, so the block flags are final too.
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -408,32 +410,32 @@ __global__ void __launch_bounds__(256) score_select_kernel(const float* __restri
   const int bh = blockIdx.y, i0 = blockIdx.x * kStripRows;
   const float* qb = qbar + static_cast<int64_t>(bh) * NB * D;
   const float* kb = kbar + static_cast<int64_t>(bh) * NB * D;
-  for (int e = tid; e < kStripRows * (D / 4); e += 256) {
+  for (int e = tid; e < kStripRows * (D / 4); e += WARPS * 32) {
     const int r = e / (D / 4), c4 = e % (D / 4);
     float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
     if (i0 + r < NB) v = __ldg(reinterpret_cast<const float4*>(qb + static_cast<int64_t>(i0 + r) * D) + c4);
     *reinterpret_cast<float4*>(sq + r * PITCH + c4 * 4) = v;
   }
   __syncthreads();
-  for (int j0 = warp * 32; j0 < NB; j0 += 8 * 32) {
-    float acc[4][4];
+  for (int j0 = warp * CHUNK; j0 < NB; j0 += WARPS * CHUNK) {
+    float acc[NT][4];
 #pragma unroll
-    for (int ni = 0; ni < 4; ni++)
+    for (int ni = 0; ni < NT; ni++)
 #pragma unroll
       for (int r = 0; r < 4; r++) acc[ni][r] = 0.f;
-    const float* krow[4];
-    bool kvalid[4];
+    const float* krow[NT];
+    bool kvalid[NT];
 #pragma unroll
-    for (int ni = 0; ni < 4; ni++) {
+    for (int ni = 0; ni < NT; ni++) {
       const int col = j0 + ni * 8 + g;
       kvalid[ni] = col < NB;
       krow[ni] = kb + static_cast<int64_t>(kvalid[ni] ? col : 0) * D + 4 * t;
     }
 #pragma unroll 4
     for (int jg = 0; jg < D / 16; jg++) {
-      float4 kv[4];
+      float4 kv[NT];
 #pragma unroll
-      for (int ni = 0; ni < 4; ni++) {
+      for (int ni = 0; ni < NT; ni++) {
         kv[ni] = make_float4(0.f, 0.f, 0.f, 0.f);
         if (kvalid[ni]) kv[ni] = __ldg(reinterpret_cast<const float4*>(krow[ni] + 16 * jg));
       }
@@ -450,7 +452,7 @@ __global__ void __launch_bounds__(256) score_select_kernel(const float* __restri
       split_tf32(qa.w, ah[1][2], al[1][2]);
       split_tf32(qc.w, ah[1][3], al[1][3]);
 #pragma unroll
-      for (int ni = 0; ni < 4; ni++) {
+      for (int ni = 0; ni < NT; ni++) {
         uint32_t bhh[2][2], bl[2][2];
         split_tf32(kv[ni].x, bhh[0][0], bl[0][0]);
         split_tf32(kv[ni].y, bhh[0][1], bl[0][1]);
@@ -465,7 +467,7 @@ __global__ void __launch_bounds__(256) score_select_kernel(const float* __restri
       }
     }
 #pragma unroll
-    for (int ni = 0; ni < 4; ni++) {
+    for (int ni = 0; ni < NT; ni++) {
       const int j = j0 + ni * 8 + 2 * t;
       *reinterpret_cast<float2*>(strip + g * SP + j) = make_float2(acc[ni][0] * scale, acc[ni][1] * scale);
       *reinterpret_cast<float2*>(strip + (g + 8) * SP + j) = make_float2(acc[ni][2] * scale, acc[ni][3] * scale);
@@ -475,8 +477,8 @@ __global__ void __launch_bounds__(256) score_select_kernel(const float* __restri
   const int b = bh / H;
   const uint8_t* pb = prot_blk + static_cast<int64_t>(b) * NB;
 #pragma unroll 1
-  for (int rr = 0; rr < kStripRows / 8; rr++) {
-    const int r = warp * (kStripRows / 8) + rr;
+  for (int rr = 0; rr < kStripRows / WARPS; rr++) {
+    const int r = warp * (kStripRows / WARPS) + rr;
     const int qi = i0 + r;
     if (qi >= NB) break;
     const int64_t row = static_cast<int64_t>(bh) * NB + qi;
@@ -518,34 +520,34 @@ __global__ void __launch_bounds__(256) expand_blocks_kernel(const uint8_t* __res
   prot_tok[idx] = prot_blk[b * NB + i / blk];
 }
 
-// Launches the fused score + list kernel with the key slots per lane that NB needs.
+// Launches the fused score + list kernel with the key slots per lane that NB needs.  Eight warps per strip (two
+// rows each): sixteen warps with one row each shorten a CTA's own latency chain, but the 512-thread CTAs, staged
+// while the pooling grid drains, took thread slots from its last CTAs and the call came out slower (0.118 against
+// 0.103 ms on the Ovi-class shape).
+template <int D, int KPL, int WARPS>
+static cudaError_t launch_score_select_as(cudaLaunchConfig_t& cfg, int NB, const float* qbar, const float* kbar,
+                                          float* bs, const uint8_t* pblk, int H, float scale, int k_keep, int pr, int pc,
+                                          int32_t* col_idx, int32_t* col_cnt) {
+  cfg.blockDim = dim3(WARPS * 32, 1, 1);
+  cfg.dynamicSmemBytes = (static_cast<size_t>(kStripRows) * (D + 4) + static_cast<size_t>(kStripRows) * strip_pitch<D>(NB)) *
+                             sizeof(float) + WARPS * 256 * sizeof(int);
+  // always the same limit (the largest NB the call accepts), so concurrent callers never race on its value
+  constexpr int kMaxSmem = (kStripRows * (D + 4) + kStripRows * strip_pitch<D>(kMaxBlocksPerRow)) * 4 + WARPS * 256 * 4;
+  cudaError_t e = cudaFuncSetAttribute(score_select_kernel<D, KPL, WARPS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       kMaxSmem);
+  if (e != cudaSuccess) return e;
+  return cudaLaunchKernelEx(&cfg, score_select_kernel<D, KPL, WARPS>, qbar, kbar, bs, pblk, H, NB, scale, k_keep, pr, pc,
+                            col_idx, col_cnt);
+}
 template <int D>
 static cudaError_t launch_score_select(cudaLaunchConfig_t& cfg, int NB, const float* qbar, const float* kbar, float* bs,
                                        const uint8_t* pblk, int H, float scale, int k_keep, int pr, int pc,
                                        int32_t* col_idx, int32_t* col_cnt) {
-  const size_t smem = (static_cast<size_t>(kStripRows) * (D + 4) + static_cast<size_t>(kStripRows) * strip_pitch<D>(NB)) *
-                          sizeof(float) + 8 * 256 * sizeof(int);
-  cfg.blockDim = dim3(256, 1, 1);
-  cfg.dynamicSmemBytes = smem;
-  // always the same limit (the largest NB the call accepts), so concurrent callers never race on its value
-  constexpr int kMaxSmem = (kStripRows * (D + 4) + kStripRows * strip_pitch<D>(kMaxBlocksPerRow)) * 4 + 8 * 256 * 4;
-  cudaError_t e;
-  if (NB <= 256) {
-    e = cudaFuncSetAttribute(score_select_kernel<D, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
-    if (e != cudaSuccess) return e;
-    return cudaLaunchKernelEx(&cfg, score_select_kernel<D, 8>, qbar, kbar, bs, pblk, H, NB, scale, k_keep, pr, pc, col_idx,
-                              col_cnt);
-  }
-  if (NB <= 512) {
-    e = cudaFuncSetAttribute(score_select_kernel<D, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
-    if (e != cudaSuccess) return e;
-    return cudaLaunchKernelEx(&cfg, score_select_kernel<D, 16>, qbar, kbar, bs, pblk, H, NB, scale, k_keep, pr, pc,
-                              col_idx, col_cnt);
-  }
-  e = cudaFuncSetAttribute(score_select_kernel<D, 64>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxSmem);
-  if (e != cudaSuccess) return e;
-  return cudaLaunchKernelEx(&cfg, score_select_kernel<D, 64>, qbar, kbar, bs, pblk, H, NB, scale, k_keep, pr, pc, col_idx,
-                            col_cnt);
+  if (NB <= 256)
+    return launch_score_select_as<D, 8, 8>(cfg, NB, qbar, kbar, bs, pblk, H, scale, k_keep, pr, pc, col_idx, col_cnt);
+  if (NB <= 512)
+    return launch_score_select_as<D, 16, 8>(cfg, NB, qbar, kbar, bs, pblk, H, scale, k_keep, pr, pc, col_idx, col_cnt);
+  return launch_score_select_as<D, 64, 8>(cfg, NB, qbar, kbar, bs, pblk, H, scale, k_keep, pr, pc, col_idx, col_cnt);
 }
 
 // The staged token select may use up to kSelectSmemKeys keys of dynamic shared memory.  The limit is always set
