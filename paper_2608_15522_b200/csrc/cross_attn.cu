@@ -461,6 +461,37 @@ __global__ void __launch_bounds__(256) head_sum_kernel(const float* __restrict__
   scores[idx] = out;
 }
 
+// The same sum for few keys and many partial slots (the reverse direction: at most 512 keys, two slots per CTA of the
+// score pass): one warp per key.  Lane l adds the terms j = l, l + 32, ... in ascending order, then the 32 lane sums
+// are combined by a fixed butterfly, so the result is reproducible bit for bit (the order differs from the kernel
+// above, which serves the other direction).
+__global__ void __launch_bounds__(256) head_sum_wide_kernel(const float* __restrict__ partial, int NCH, int B, int H,
+                                                            int Nk, float beta, float gamma, float* __restrict__ scores) {
+  const int64_t idx = static_cast<int64_t>(blockIdx.x) * 8 + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (idx >= static_cast<int64_t>(B) * Nk) return;
+  const int b = static_cast<int>(idx / Nk), i = static_cast<int>(idx % Nk);
+  const int J = H * NCH;
+  float acc = 0.f;
+  for (int j0 = lane; j0 < J; j0 += 32 * 4) {
+    float v[4];
+#pragma unroll
+    for (int u = 0; u < 4; u++) {
+      const int j = j0 + 32 * u, h = j / NCH, ch = j % NCH;
+      v[u] = (j < J) ? partial[(static_cast<int64_t>(ch) * B * H + static_cast<int64_t>(b) * H + h) * Nk + i] : 0.f;
+    }
+#pragma unroll
+    for (int u = 0; u < 4; u++) acc += v[u];
+  }
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+  if (lane == 0) {
+    float out = gamma * acc;
+    if (beta != 0.f) out = fmaf(beta, scores[idx], out);
+    scores[idx] = out;
+  }
+}
+
 struct CrossPlan {
   int blk, NQT, NKB, n_split, tps;           // pass 1 (key tiles of blk)
   int NKT, NCH, W, n_range, tpr;             // pass 2 (key tiles of 128)
@@ -603,8 +634,8 @@ static int run_cross(int B, int H, int Nq, int Nk, const avsa_bf16_4d& q, const 
     rp.scale_log2 = scale * 1.4426950408889634f;
     colsum_rev_kernel<D><<<dim3(c.rev_ranges, H, B), kColThreads, smem, st>>>(tq, tk, rp);
     const int64_t n = static_cast<int64_t>(B) * Nk;
-    head_sum_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, st>>>(partial, c.rev_slots, B, H, Nk, beta, gamma,
-                                                                           scores);
+    head_sum_wide_kernel<<<static_cast<unsigned>((n + 7) / 8), 256, 0, st>>>(partial, c.rev_slots, B, H, Nk, beta, gamma,
+                                                                            scores);
   }
   // ---- pass 2, queries resident (at most 512 queries)
   if (scores != nullptr && !c.reverse) {
