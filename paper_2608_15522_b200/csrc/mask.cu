@@ -87,10 +87,11 @@ __global__ void __launch_bounds__(256) pool_kernel(const __nv_bfloat16* __restri
 // (x = hi + lo exactly to 2^-22) and three products a_lo*b_hi + a_hi*b_lo + a_hi*b_hi are accumulated in
 // fp32 (m16n8k8 MMAs; the block-score problem is far too small for the tcgen05 path).
 // ------------------------------------------------------------------------------------------------
+// hi = x with the 13 mantissa bits cleared that a tf32 operand does not have, lo = x - hi (exact in fp32; the MMA
+// reads its leading 10 mantissa bits, which leaves an error of 2^-21 |x|)
 __device__ __forceinline__ void split_tf32(float x, uint32_t& hi, uint32_t& lo) {
-  asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(hi) : "f"(x));
-  const float r = x - __uint_as_float(hi);
-  asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(lo) : "f"(r));
+  hi = __float_as_uint(x) & 0xffffe000u;
+  lo = __float_as_uint(x - __uint_as_float(hi));
 }
 __device__ __forceinline__ void mma_tf32(float (&d)[4], const uint32_t (&a)[4], const uint32_t (&b)[2]) {
   asm volatile(
@@ -288,24 +289,25 @@ __device__ __forceinline__ void select_row(const float* src, const uint8_t* __re
     want = k_keep;
     for (int pass = 0; pass < 4; pass++) {
       const int shift = 24 - 8 * pass;
-      // digit range of the keys still in play: when they all share the digit (typical for the leading byte)
-      // the pass needs no histogram at all
-      uint32_t dmin = 255u, dmax = 0u;
+      // digit range of the keys: when they all share the leading byte (sign and high exponent bits: the usual
+      // case) the first pass needs no histogram at all; later bytes hardly ever agree, so only it is checked
+      if (pass == 0) {
+        uint32_t dmin = 255u, dmax = 0u;
 #pragma unroll
-      for (int j = 0; j < KPL; j++) {
-        const bool in = (j * 32 + lane < NB) && ((keys[j] & mask) == prefix);
-        const uint32_t dg = (keys[j] >> shift) & 255u;
-        if (in) {
-          dmin = min(dmin, dg);
-          dmax = max(dmax, dg);
+        for (int j = 0; j < KPL; j++) {
+          const uint32_t dg = keys[j] >> 24;
+          if (j * 32 + lane < NB) {
+            dmin = min(dmin, dg);
+            dmax = max(dmax, dg);
+          }
         }
-      }
-      dmin = __reduce_min_sync(0xffffffffu, dmin);
-      dmax = __reduce_max_sync(0xffffffffu, dmax);
-      if (dmin == dmax) {
-        prefix |= dmin << shift;
-        mask |= 255u << shift;
-        continue;
+        dmin = __reduce_min_sync(0xffffffffu, dmin);
+        dmax = __reduce_max_sync(0xffffffffu, dmax);
+        if (dmin == dmax) {
+          prefix = dmin << 24;
+          mask = 255u << 24;
+          continue;
+        }
       }
 #pragma unroll
       for (int i = 0; i < 8; i++) bins[i * 32 + lane] = 0;
@@ -397,9 +399,10 @@ __global__ void __launch_bounds__(WARPS * 32) score_select_kernel(const float* _
   constexpr int NT = 32 / WARPS;              // 8-column MMA tiles per warp and pass: 4 with 8 warps, 2 with 16
   constexpr int CHUNK = NT * 8;               // columns per warp and pass
   extern __shared__ __align__(16) float strip_smem[];
-  float* sq = strip_smem;                                   // [16][PITCH] pooled queries of the strip
+  uint32_t* sq_hi = reinterpret_cast<uint32_t*>(strip_smem);            // [16][PITCH] pooled queries of the strip,
+  uint32_t* sq_lo = sq_hi + kStripRows * PITCH;                          // split into their two tf32 halves once
   const int SP = strip_pitch<D>(NB);
-  float* strip = sq + kStripRows * PITCH;                   // [16][SP] block scores of the strip
+  float* strip = strip_smem + 2 * kStripRows * PITCH;       // [16][SP] block scores of the strip
   int* all_bins = reinterpret_cast<int*>(strip + kStripRows * SP);      // [WARPS][256]
   // Staged behind the pooling grid (programmatic dependent launch) and waits for it here; the pooling grid in
   // turn retires only after the token select, so the block flags are final too.
@@ -414,7 +417,13 @@ __global__ void __launch_bounds__(WARPS * 32) score_select_kernel(const float* _
     const int r = e / (D / 4), c4 = e % (D / 4);
     float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
     if (i0 + r < NB) v = __ldg(reinterpret_cast<const float4*>(qb + static_cast<int64_t>(i0 + r) * D) + c4);
-    *reinterpret_cast<float4*>(sq + r * PITCH + c4 * 4) = v;
+    uint4 vh, vl;
+    split_tf32(v.x, vh.x, vl.x);
+    split_tf32(v.y, vh.y, vl.y);
+    split_tf32(v.z, vh.z, vl.z);
+    split_tf32(v.w, vh.w, vl.w);
+    *reinterpret_cast<uint4*>(sq_hi + r * PITCH + c4 * 4) = vh;
+    *reinterpret_cast<uint4*>(sq_lo + r * PITCH + c4 * 4) = vl;
   }
   __syncthreads();
   for (int j0 = warp * CHUNK; j0 < NB; j0 += WARPS * CHUNK) {
@@ -439,18 +448,13 @@ __global__ void __launch_bounds__(WARPS * 32) score_select_kernel(const float* _
         kv[ni] = make_float4(0.f, 0.f, 0.f, 0.f);
         if (kvalid[ni]) kv[ni] = __ldg(reinterpret_cast<const float4*>(krow[ni] + 16 * jg));
       }
-      const float4 qa = *reinterpret_cast<const float4*>(sq + g * PITCH + 16 * jg + 4 * t);
-      const float4 qc = *reinterpret_cast<const float4*>(sq + (g + 8) * PITCH + 16 * jg + 4 * t);
+      const uint4 qah = *reinterpret_cast<const uint4*>(sq_hi + g * PITCH + 16 * jg + 4 * t);
+      const uint4 qal = *reinterpret_cast<const uint4*>(sq_lo + g * PITCH + 16 * jg + 4 * t);
+      const uint4 qch = *reinterpret_cast<const uint4*>(sq_hi + (g + 8) * PITCH + 16 * jg + 4 * t);
+      const uint4 qcl = *reinterpret_cast<const uint4*>(sq_lo + (g + 8) * PITCH + 16 * jg + 4 * t);
       // two k-steps: (x, y) and (z, w) of each piece
-      uint32_t ah[2][4], al[2][4];
-      split_tf32(qa.x, ah[0][0], al[0][0]);
-      split_tf32(qc.x, ah[0][1], al[0][1]);
-      split_tf32(qa.y, ah[0][2], al[0][2]);
-      split_tf32(qc.y, ah[0][3], al[0][3]);
-      split_tf32(qa.z, ah[1][0], al[1][0]);
-      split_tf32(qc.z, ah[1][1], al[1][1]);
-      split_tf32(qa.w, ah[1][2], al[1][2]);
-      split_tf32(qc.w, ah[1][3], al[1][3]);
+      const uint32_t ah[2][4] = {{qah.x, qch.x, qah.y, qch.y}, {qah.z, qch.z, qah.w, qch.w}};
+      const uint32_t al[2][4] = {{qal.x, qcl.x, qal.y, qcl.y}, {qal.z, qcl.z, qal.w, qcl.w}};
 #pragma unroll
       for (int ni = 0; ni < NT; ni++) {
         uint32_t bhh[2][2], bl[2][2];
@@ -529,10 +533,10 @@ static cudaError_t launch_score_select_as(cudaLaunchConfig_t& cfg, int NB, const
                                           float* bs, const uint8_t* pblk, int H, float scale, int k_keep, int pr, int pc,
                                           int32_t* col_idx, int32_t* col_cnt) {
   cfg.blockDim = dim3(WARPS * 32, 1, 1);
-  cfg.dynamicSmemBytes = (static_cast<size_t>(kStripRows) * (D + 4) + static_cast<size_t>(kStripRows) * strip_pitch<D>(NB)) *
+  cfg.dynamicSmemBytes = (static_cast<size_t>(2 * kStripRows) * (D + 4) + static_cast<size_t>(kStripRows) * strip_pitch<D>(NB)) *
                              sizeof(float) + WARPS * 256 * sizeof(int);
   // always the same limit (the largest NB the call accepts), so concurrent callers never race on its value
-  constexpr int kMaxSmem = (kStripRows * (D + 4) + kStripRows * strip_pitch<D>(kMaxBlocksPerRow)) * 4 + WARPS * 256 * 4;
+  constexpr int kMaxSmem = (2 * kStripRows * (D + 4) + kStripRows * strip_pitch<D>(kMaxBlocksPerRow)) * 4 + WARPS * 256 * 4;
   cudaError_t e = cudaFuncSetAttribute(score_select_kernel<D, KPL, WARPS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        kMaxSmem);
   if (e != cudaSuccess) return e;
