@@ -10,7 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libavsa.so")
 SOURCES = ["api.cu", "mask.cu", "sparse_attn.cu", "cross_attn.cu", "protected_rows.cu", "cache_indicators.cu"]
-HEADERS = ["avsa_common.cuh", "sm100_ptx.cuh", "attn_kernel.cuh", "attn_persist_kernel.cuh", os.path.join("..", "..", "include", "avsa.h")]
+HEADERS = sorted(f for f in os.listdir(CSRC) if f.endswith(".cuh")) + [os.path.join("..", "..", "include", "avsa.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden"]
 

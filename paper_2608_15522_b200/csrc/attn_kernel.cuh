@@ -24,6 +24,12 @@
 namespace avsa {
 
 constexpr int kAttnThreads = 384;
+// Register reallocation between the roles (setmaxnreg): a CTA is launched with 384 x 168 = 64512 registers; afterwards
+// its four service warps hold 64 each and its eight softmax warps 216: 128 x 64 + 256 x 216 = 63488.  A request
+// beyond what the CTA holds makes setmaxnreg.inc wait for ever, which no time-limited barrier catches: the sum has
+// to stay below the launch figure.
+constexpr int kLaunchRegs = 168, kServiceRegs = 64, kSoftmaxRegs = 216;
+static_assert(4 * 32 * kServiceRegs + 8 * 32 * kSoftmaxRegs <= kAttnThreads * kLaunchRegs, "setmaxnreg budget exceeded");
 constexpr int kStages = 3;
 constexpr float kRescaleThreshold = 8.0f;   // log2 units: O is rescaled only when a row max grew by more
 
