@@ -187,6 +187,31 @@ def test_block_scores_and_selection_from_pooled_qk(name):
                 assert want[b, h, i, kept].min() >= want[b, h, i, rest].max() - tol
 
 
+@pytest.mark.parametrize("d,nb,tail", [(128, 520, 5), (64, 300, 17), (128, 33, 0)])
+def test_block_scores_and_lists_long_rows(d, nb, tail):
+    """Rows of more than 256 and more than 512 key blocks (more keys per lane in the select, larger strips in shared
+    memory), a ragged last block, and a block count that is no multiple of the 16-row strip: pooled block scores
+    against the oracle, lists bit-exact given those scores."""
+    blk = d
+    N = blk * (nb - 1) + (tail if tail else blk)
+    B, H = 1, 2
+    g = torch.Generator().manual_seed(nb)
+    q = torch.randn((B, H, N, d), generator=g).bfloat16()
+    k = (torch.randn((B, H, N, d), generator=g) + 0.5).bfloat16()
+    s = torch.rand((B, N), generator=g)
+    n_protect, k_keep = N // 50, max(1, nb // 5)
+    out = av.avsa_build_block_mask(q.cuda(), k.cuda(), s.cuda(), n_protect, k_keep, blk)
+    _status_ok(out["ws"])
+    got = out["block_scores"].cpu().numpy()
+    want = orc.block_scores(_np64(q), _np64(k), blk)
+    assert got.shape == (B, H, nb, nb)
+    assert np.abs(got - want).max() <= 1e-4 * max(1.0, np.abs(want).max())
+    idx, cnt, ptok, pblk = orc.build_block_mask(got, s.numpy(), n_protect, k_keep, blk, N)
+    assert np.array_equal(out["col_cnt"].cpu().numpy(), cnt)
+    assert np.array_equal(out["col_idx"].cpu().numpy(), idx)
+    assert np.array_equal(out["prot_tok"].cpu().numpy(), ptok) and np.array_equal(out["prot_blk"].cpu().numpy(), pblk)
+
+
 # ------------------------------------------------------------------------------------------- sparse attention
 def _run_sparse_case(w, seed, idx, cnt, want_lse=True):
     q, k, v = wl.make_self_qkv(w, seed)
