@@ -37,7 +37,7 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # summarised under profiles/ (None until a capture exists for that workload)
 NCU_TRAFFIC_BYTES = {"mid": 482.3e6,      # captured (profiles/attn_persist_kernel_mid.md)
                      "ovi": 861.1e6}      # captured on the full launch with the two DRAM counters only (same file)
-KERNELS_PER_STEP = 12   # cross: clear, pass 1, its redo pass, merge, pass 2, head sum; mask: select, pool, scores + lists; attn: prep, persistent, redo
+KERNELS_PER_STEP = 11   # cross: clear, pass 1, its redo pass, pass 2, head sum + merge; mask: select, pool, scores + lists; attn: prep, persistent, redo
 
 
 def load_peaks():

@@ -500,16 +500,17 @@ attn_redo_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant_
 // With a row map the result of compact row r goes to row row_map[b][r] of the output (rows mapped to
 // a negative index are skipped): that is how recomputed protected rows are scattered back.
 // ------------------------------------------------------------------------------------------------
+// (`block`, `tid`: index of a group of 128 threads and the thread's place in it, so that another kernel can run
+// this work in part of its grid)
 template <int BLK, int D>
-__global__ void __launch_bounds__(128) merge_splits_kernel(const float* __restrict__ part_o,
-                                                           const float* __restrict__ part_lse2, int n_split, int NQT,
-                                                           int Nq, int H, int total_rows, __nv_bfloat16* __restrict__ o,
-                                                           int64_t o_sb, int64_t o_sh, int64_t o_sn,
-                                                           float* __restrict__ lse, const int32_t* __restrict__ row_map,
-                                                           int row_map_stride, int n_out) {
+__device__ __forceinline__ void merge_splits_rows(int block, int tid, const float* __restrict__ part_o,
+                                                  const float* __restrict__ part_lse2, int n_split, int NQT, int Nq,
+                                                  int H, int total_rows, __nv_bfloat16* __restrict__ o, int64_t o_sb,
+                                                  int64_t o_sh, int64_t o_sn, float* __restrict__ lse,
+                                                  const int32_t* __restrict__ row_map, int row_map_stride, int n_out) {
   constexpr int TPR = D / 4;
-  const int rg = blockIdx.x * (128 / TPR) + threadIdx.x / TPR;
-  const int c4 = threadIdx.x % TPR;
+  const int rg = block * (128 / TPR) + tid / TPR;
+  const int c4 = tid % TPR;
   if (rg >= total_rows) return;
   const int bh = rg / Nq, qrow = rg % Nq;
   const int b = bh / H, h = bh % H;
@@ -541,6 +542,17 @@ __global__ void __launch_bounds__(128) merge_splits_kernel(const float* __restri
     *reinterpret_cast<uint2*>(o + b * o_sb + h * o_sh + out_row * o_sn + c4 * 4) = pk;
   }
   if (c4 == 0 && lse != nullptr) lse[static_cast<int64_t>(bh) * n_out + out_row] = (M + log2f(W)) * 0.6931471805599453f;
+}
+
+template <int BLK, int D>
+__global__ void __launch_bounds__(128) merge_splits_kernel(const float* __restrict__ part_o,
+                                                           const float* __restrict__ part_lse2, int n_split, int NQT,
+                                                           int Nq, int H, int total_rows, __nv_bfloat16* __restrict__ o,
+                                                           int64_t o_sb, int64_t o_sh, int64_t o_sn,
+                                                           float* __restrict__ lse, const int32_t* __restrict__ row_map,
+                                                           int row_map_stride, int n_out) {
+  merge_splits_rows<BLK, D>(blockIdx.x, threadIdx.x, part_o, part_lse2, n_split, NQT, Nq, H, total_rows, o, o_sb, o_sh,
+                            o_sn, lse, row_map, row_map_stride, n_out);
 }
 
 }  // namespace avsa

@@ -19,7 +19,9 @@ constexpr int kColThreads = 384;
 constexpr int kColStages = 3;
 
 struct ColsumParams {
-  const float* lse;        // [B,H,Nq] natural log
+  const float* lse;        // [B,H,Nq] natural log; used when part_lse2 is null
+  const float* part_lse2;  // or the log2-domain LSEs of pass 1's key splits, [B,H,NQT,n_split,blk], merged here
+  int n_split, NQT, blk;
   float* partial;          // [NCH][B,H,Nk]
   StatusRecord* status;
   int H, Nq, Nk, NKT;      // NKT = key tiles of 128
@@ -84,8 +86,25 @@ colsum_kernel(const __grid_constant__ CUtensorMap tmq, const __grid_constant__ C
     prefetch_tmap(&tmk);
   }
   // negated log2-domain LSEs (one packed FMA then gives s*c - lse2); queries beyond Nq get -inf: exp2 = 0
-  for (int j = tid; j < NCH * W; j += kColThreads)
-    lse2[j] = (j < p.Nq) ? -p.lse[(static_cast<int64_t>(b) * p.H + h) * p.Nq + j] * 1.4426950408889634f : -INFINITY;
+  // (straight from the splits' partial LSEs when pass 1 left its merge for later: the same maximum-and-sum as the
+  // merge kernel, in the log2 domain)
+  for (int j = tid; j < NCH * W; j += kColThreads) {
+    float v = -INFINITY;
+    if (j < p.Nq) {
+      if (p.part_lse2 != nullptr) {
+        const int64_t item0 = ((static_cast<int64_t>(b) * p.H + h) * p.NQT + j / p.blk) * p.n_split;
+        const float* pl = p.part_lse2 + item0 * p.blk + j % p.blk;
+        float M = -INFINITY;
+        for (int s = 0; s < p.n_split; s++) M = fmaxf(M, pl[s * p.blk]);
+        float Wsum = 0.f;
+        for (int s = 0; s < p.n_split; s++) Wsum += exp2f(pl[s * p.blk] - M);
+        v = -(M + log2f(Wsum));
+      } else {
+        v = -p.lse[(static_cast<int64_t>(b) * p.H + h) * p.Nq + j] * 1.4426950408889634f;
+      }
+    }
+    lse2[j] = v;
+  }
   if (warp == 2) {
     tmem_alloc(smem_u32(const_cast<uint32_t*>(misc)), 512);
     tmem_relinquish();
@@ -436,9 +455,9 @@ __global__ void __launch_bounds__(256) lse_to_log2_kernel(const float* __restric
 }
 
 // scores[b,i] = beta * scores[b,i] + gamma * sum_h sum_ch partial[ch][b,h,i], heads in ascending order
-__global__ void __launch_bounds__(256) head_sum_kernel(const float* __restrict__ partial, int NCH, int B, int H,
-                                                       int Nk, float beta, float gamma, float* __restrict__ scores) {
-  const int64_t idx = static_cast<int64_t>(blockIdx.x) * 256 + threadIdx.x;
+__device__ __forceinline__ void head_sum_keys(int block, int tid, const float* __restrict__ partial, int NCH, int B,
+                                              int H, int Nk, float beta, float gamma, float* __restrict__ scores) {
+  const int64_t idx = static_cast<int64_t>(block) * 256 + tid;
   if (idx >= static_cast<int64_t>(B) * Nk) return;
   const int b = static_cast<int>(idx / Nk), i = static_cast<int>(idx % Nk);
   // Fixed summation order: head major, partial slot minor.  Eight loads are issued together (a plain loop made
@@ -459,6 +478,30 @@ __global__ void __launch_bounds__(256) head_sum_kernel(const float* __restrict__
   float out = gamma * acc;
   if (beta != 0.f) out = fmaf(beta, scores[idx], out);
   scores[idx] = out;
+}
+__global__ void __launch_bounds__(256) head_sum_kernel(const float* __restrict__ partial, int NCH, int B, int H,
+                                                       int Nk, float beta, float gamma, float* __restrict__ scores) {
+  head_sum_keys(blockIdx.x, threadIdx.x, partial, NCH, B, H, Nk, beta, gamma, scores);
+}
+
+// End of the forward call in one grid: the first `hs_blocks` CTAs sum the score partials over heads, the rest merge
+// the key splits of pass 1 into O and the LSE (two groups of 128 threads per CTA).  The score pass merged the LSEs
+// it needs by itself, so nothing waits for this merge.
+template <int BLK, int D>
+__global__ void __launch_bounds__(256) cross_finalize_kernel(int hs_blocks, const float* __restrict__ partial, int NCH, int B,
+                                                             int H, int Nk, float beta, float gamma,
+                                                             float* __restrict__ scores, const float* __restrict__ part_o,
+                                                             const float* __restrict__ part_lse2, int n_split, int NQT,
+                                                             int Nq, int total_rows, __nv_bfloat16* __restrict__ o,
+                                                             int64_t o_sb, int64_t o_sh, int64_t o_sn,
+                                                             float* __restrict__ lse) {
+  if (static_cast<int>(blockIdx.x) < hs_blocks) {
+    head_sum_keys(blockIdx.x, threadIdx.x, partial, NCH, B, H, Nk, beta, gamma, scores);
+  } else {
+    const int block = (static_cast<int>(blockIdx.x) - hs_blocks) * 2 + (threadIdx.x >> 7);
+    merge_splits_rows<BLK, D>(block, threadIdx.x & 127, part_o, part_lse2, n_split, NQT, Nq, H, total_rows, o, o_sb, o_sh,
+                              o_sn, lse, nullptr, 0, Nq);
+  }
 }
 
 // The same sum for few keys and many partial slots (the reverse direction: at most 512 keys, two slots per CTA of the
@@ -553,6 +596,7 @@ static int run_cross(int B, int H, int Nq, int Nk, const avsa_bf16_4d& q, const 
   float* lse = lse_out != nullptr ? lse_out : reinterpret_cast<float*>(ws + c.off_lse);
   float* partial = reinterpret_cast<float*>(ws + c.off_partial);
   clear_status_kernel<<<1, 1, 0, st>>>(status);
+  bool merge_late = false;
   // ---- pass 1
   {
     using L = AttnSmem<BLK, D>;
@@ -602,11 +646,14 @@ static int run_cross(int B, int H, int Nq, int Nk, const avsa_bf16_4d& q, const 
       attn_persist_kernel<BLK, D, MODE_RANGE><<<pgrid, kAttnThreads, LP::kTotal, st>>>(tq, tk, tv, tq, prm, redo, nullptr,
                                                                                        static_cast<int>(items));
       attn_redo_kernel<BLK, D, MODE_RANGE><<<pgrid, kAttnThreads, L::kTotal, st>>>(tq, tk, tv, tq, prm, redo);
-      const int total_rows = B * H * Nq;
-      constexpr int RPB = 128 / (D / 4);
-      merge_splits_kernel<BLK, D><<<(total_rows + RPB - 1) / RPB, 128, 0, st>>>(
-          part_o, part_lse, c.n_split, c.NQT, Nq, H, total_rows, static_cast<__nv_bfloat16*>(o), q.stride_b, q.stride_h,
-          q.stride_n, lse, nullptr, 0, Nq);
+      merge_late = scores != nullptr && !c.reverse;      // then the merge rides in the call's last grid
+      if (!merge_late) {
+        const int total_rows = B * H * Nq;
+        constexpr int RPB = 128 / (D / 4);
+        merge_splits_kernel<BLK, D><<<(total_rows + RPB - 1) / RPB, 128, 0, st>>>(
+            part_o, part_lse, c.n_split, c.NQT, Nq, H, total_rows, static_cast<__nv_bfloat16*>(o), q.stride_b, q.stride_h,
+            q.stride_n, lse, nullptr, 0, Nq);
+      }
     }
   }
   // ---- pass 2, keys resident (many queries, at most 512 keys)
@@ -648,6 +695,10 @@ static int run_cross(int B, int H, int Nq, int Nk, const avsa_bf16_4d& q, const 
       return AVSA_ERR_CUDA;
     ColsumParams cp;
     cp.lse = lse;
+    cp.part_lse2 = merge_late ? part_lse : nullptr;
+    cp.n_split = c.n_split;
+    cp.NQT = c.NQT;
+    cp.blk = c.blk;
     cp.partial = partial;
     cp.status = status;
     cp.H = H;
@@ -662,8 +713,17 @@ static int run_cross(int B, int H, int Nq, int Nk, const avsa_bf16_4d& q, const 
     dim3 grid(c.n_range, H, B);
     colsum_kernel<D><<<grid, kColThreads, smem, st>>>(tq, tk, cp);
     const int64_t n = static_cast<int64_t>(B) * Nk;
-    head_sum_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, st>>>(partial, c.NCH, B, H, Nk, beta, gamma,
-                                                                           scores);
+    const int hs_blocks = static_cast<int>((n + 255) / 256);
+    if (merge_late) {
+      const int total_rows = B * H * Nq;
+      constexpr int RPB = 128 / (D / 4);
+      const int merge_blocks = ((total_rows + RPB - 1) / RPB + 1) / 2;
+      cross_finalize_kernel<BLK, D><<<hs_blocks + merge_blocks, 256, 0, st>>>(
+          hs_blocks, partial, c.NCH, B, H, Nk, beta, gamma, scores, part_o, part_lse, c.n_split, c.NQT, Nq, total_rows,
+          static_cast<__nv_bfloat16*>(o), q.stride_b, q.stride_h, q.stride_n, lse);
+    } else {
+      head_sum_kernel<<<hs_blocks, 256, 0, st>>>(partial, c.NCH, B, H, Nk, beta, gamma, scores);
+    }
   }
   return cudaGetLastError() == cudaSuccess ? AVSA_OK : AVSA_ERR_CUDA;
 }
