@@ -89,6 +89,9 @@ __global__ void __launch_bounds__(256) pool_kernel(const __nv_bfloat16* __restri
 // ------------------------------------------------------------------------------------------------
 // hi = x with the 13 mantissa bits cleared that a tf32 operand does not have, lo = x - hi (exact in fp32; the MMA
 // reads its leading 10 mantissa bits, which leaves an error of 2^-21 |x|)
+__device__ __forceinline__ uint32_t smem_u32_of(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
 __device__ __forceinline__ void split_tf32(float x, uint32_t& hi, uint32_t& lo) {
   hi = __float_as_uint(x) & 0xffffe000u;
   lo = __float_as_uint(x - __uint_as_float(hi));
@@ -404,6 +407,8 @@ __global__ void __launch_bounds__(WARPS * 32) score_select_kernel(const float* _
   const int SP = strip_pitch<D>(NB);
   float* strip = strip_smem + 2 * kStripRows * PITCH;       // [16][SP] block scores of the strip
   int* all_bins = reinterpret_cast<int*>(strip + kStripRows * SP);      // [WARPS][256]
+  float4* ring = reinterpret_cast<float4*>(all_bins + WARPS * 256);     // [WARPS][4 slots][2 tiles][32 lanes]
+  static_assert(NT == 4, "the key ring holds two tile pairs per 16-channel group");
   // Staged behind the pooling grid (programmatic dependent launch) and waits for it here; the pooling grid in
   // turn retires only after the token select, so the block flags are final too.
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -413,6 +418,32 @@ __global__ void __launch_bounds__(WARPS * 32) score_select_kernel(const float* _
   const int bh = blockIdx.y, i0 = blockIdx.x * kStripRows;
   const float* qb = qbar + static_cast<int64_t>(bh) * NB * D;
   const float* kb = kbar + static_cast<int64_t>(bh) * NB * D;
+  // The pooled keys come through a ring of four 16-byte slots per lane and MMA tile pair (cp.async, no registers
+  // held): the pieces of three half-steps ahead are in flight under the MMAs of the current one, and the first
+  // three of a warp's first chunk already under the load of the strip's queries.  A plain load per step left every
+  // step waiting for its own L2 round trip (1500 cycles each, eight in a row).
+  constexpr int HS = (D / 16) * 2;            // half-steps: (16-channel group jg, tile pair hp)
+  const uint32_t ring_base = smem_u32_of(ring) + (warp * 4 * 2 * 32 + lane) * 16;
+  auto issue = [&](int j0, int hs) {
+    const int jg = hs >> 1, hp = hs & 1;
+#pragma unroll
+    for (int n2 = 0; n2 < 2; n2++) {
+      const int col = j0 + (hp * 2 + n2) * 8 + g;
+      const bool valid = col < NB;                          // beyond the last key block: zero fill
+      const float* src = kb + static_cast<int64_t>(valid ? col : 0) * D + 4 * t + 16 * jg;
+      const uint32_t dst = ring_base + (((hs & 3) * 2 + n2) * 32) * 16;
+      const int bytes = valid ? 16 : 0;
+      asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(bytes) : "memory");
+    }
+  };
+  const int j_first = warp * CHUNK;
+  if (j_first < NB) {
+#pragma unroll
+    for (int hs = 0; hs < 3; hs++) {
+      issue(j_first, hs);
+      asm volatile("cp.async.commit_group;" ::: "memory");
+    }
+  }
   for (int e = tid; e < kStripRows * (D / 4); e += WARPS * 32) {
     const int r = e / (D / 4), c4 = e % (D / 4);
     float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -432,36 +463,40 @@ __global__ void __launch_bounds__(WARPS * 32) score_select_kernel(const float* _
     for (int ni = 0; ni < NT; ni++)
 #pragma unroll
       for (int r = 0; r < 4; r++) acc[ni][r] = 0.f;
-    const float* krow[NT];
-    bool kvalid[NT];
+    if (j0 != j_first) {
 #pragma unroll
-    for (int ni = 0; ni < NT; ni++) {
-      const int col = j0 + ni * 8 + g;
-      kvalid[ni] = col < NB;
-      krow[ni] = kb + static_cast<int64_t>(kvalid[ni] ? col : 0) * D + 4 * t;
-    }
-#pragma unroll 4
-    for (int jg = 0; jg < D / 16; jg++) {
-      float4 kv[NT];
-#pragma unroll
-      for (int ni = 0; ni < NT; ni++) {
-        kv[ni] = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (kvalid[ni]) kv[ni] = __ldg(reinterpret_cast<const float4*>(krow[ni] + 16 * jg));
+      for (int hs = 0; hs < 3; hs++) {
+        issue(j0, hs);
+        asm volatile("cp.async.commit_group;" ::: "memory");
       }
-      const uint4 qah = *reinterpret_cast<const uint4*>(sq_hi + g * PITCH + 16 * jg + 4 * t);
-      const uint4 qal = *reinterpret_cast<const uint4*>(sq_lo + g * PITCH + 16 * jg + 4 * t);
-      const uint4 qch = *reinterpret_cast<const uint4*>(sq_hi + (g + 8) * PITCH + 16 * jg + 4 * t);
-      const uint4 qcl = *reinterpret_cast<const uint4*>(sq_lo + (g + 8) * PITCH + 16 * jg + 4 * t);
-      // two k-steps: (x, y) and (z, w) of each piece
-      const uint32_t ah[2][4] = {{qah.x, qch.x, qah.y, qch.y}, {qah.z, qch.z, qah.w, qch.w}};
-      const uint32_t al[2][4] = {{qal.x, qcl.x, qal.y, qcl.y}, {qal.z, qcl.z, qal.w, qcl.w}};
+    }
+    uint32_t ah[2][4], al[2][4];
 #pragma unroll
-      for (int ni = 0; ni < NT; ni++) {
+    for (int hs = 0; hs < HS; hs++) {
+      const int jg = hs >> 1, hp = hs & 1;
+      if (hs + 3 < HS) issue(j0, hs + 3);
+      asm volatile("cp.async.commit_group;" ::: "memory");      // (an empty group near the end keeps the count uniform)
+      asm volatile("cp.async.wait_group 3;" ::: "memory");       // the pieces of half-step hs have landed
+      if (hp == 0) {
+        const uint4 qah = *reinterpret_cast<const uint4*>(sq_hi + g * PITCH + 16 * jg + 4 * t);
+        const uint4 qal = *reinterpret_cast<const uint4*>(sq_lo + g * PITCH + 16 * jg + 4 * t);
+        const uint4 qch = *reinterpret_cast<const uint4*>(sq_hi + (g + 8) * PITCH + 16 * jg + 4 * t);
+        const uint4 qcl = *reinterpret_cast<const uint4*>(sq_lo + (g + 8) * PITCH + 16 * jg + 4 * t);
+        // two k-steps: (x, y) and (z, w) of each piece
+        ah[0][0] = qah.x; ah[0][1] = qch.x; ah[0][2] = qah.y; ah[0][3] = qch.y;
+        ah[1][0] = qah.z; ah[1][1] = qch.z; ah[1][2] = qah.w; ah[1][3] = qch.w;
+        al[0][0] = qal.x; al[0][1] = qcl.x; al[0][2] = qal.y; al[0][3] = qcl.y;
+        al[1][0] = qal.z; al[1][1] = qcl.z; al[1][2] = qal.w; al[1][3] = qcl.w;
+      }
+#pragma unroll
+      for (int n2 = 0; n2 < 2; n2++) {
+        const int ni = hp * 2 + n2;
+        const float4 kvp = ring[(warp * 4 * 2 + (hs & 3) * 2 + n2) * 32 + lane];
         uint32_t bhh[2][2], bl[2][2];
-        split_tf32(kv[ni].x, bhh[0][0], bl[0][0]);
-        split_tf32(kv[ni].y, bhh[0][1], bl[0][1]);
-        split_tf32(kv[ni].z, bhh[1][0], bl[1][0]);
-        split_tf32(kv[ni].w, bhh[1][1], bl[1][1]);
+        split_tf32(kvp.x, bhh[0][0], bl[0][0]);
+        split_tf32(kvp.y, bhh[0][1], bl[0][1]);
+        split_tf32(kvp.z, bhh[1][0], bl[1][0]);
+        split_tf32(kvp.w, bhh[1][1], bl[1][1]);
 #pragma unroll
         for (int s2 = 0; s2 < 2; s2++) {
           mma_tf32(acc[ni], al[s2], bhh[s2]);     // small terms first
@@ -470,6 +505,7 @@ __global__ void __launch_bounds__(WARPS * 32) score_select_kernel(const float* _
         }
       }
     }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
 #pragma unroll
     for (int ni = 0; ni < NT; ni++) {
       const int j = j0 + ni * 8 + 2 * t;
@@ -534,9 +570,9 @@ static cudaError_t launch_score_select_as(cudaLaunchConfig_t& cfg, int NB, const
                                           int32_t* col_idx, int32_t* col_cnt) {
   cfg.blockDim = dim3(WARPS * 32, 1, 1);
   cfg.dynamicSmemBytes = (static_cast<size_t>(2 * kStripRows) * (D + 4) + static_cast<size_t>(kStripRows) * strip_pitch<D>(NB)) *
-                             sizeof(float) + WARPS * 256 * sizeof(int);
+                             sizeof(float) + WARPS * 256 * sizeof(int) + WARPS * 4 * 2 * 32 * 16;
   // always the same limit (the largest NB the call accepts), so concurrent callers never race on its value
-  constexpr int kMaxSmem = (2 * kStripRows * (D + 4) + kStripRows * strip_pitch<D>(kMaxBlocksPerRow)) * 4 + WARPS * 256 * 4;
+  constexpr int kMaxSmem = (2 * kStripRows * (D + 4) + kStripRows * strip_pitch<D>(kMaxBlocksPerRow)) * 4 + WARPS * 256 * 4 + WARPS * 4 * 2 * 32 * 16;
   cudaError_t e = cudaFuncSetAttribute(score_select_kernel<D, KPL, WARPS>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        kMaxSmem);
   if (e != cudaSuccess) return e;
